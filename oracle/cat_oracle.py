@@ -1,0 +1,220 @@
+"""fp64 CPU oracle for the Confidence-Adaptive Token (CAT) loss and its gradients.
+
+THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, obviously
+correct restatement of what the paper's training objective computes, written
+from the formulas (PARD-2, Section 3.2 "Confidence-Adaptive Token Optimization
+Strategy", Eq. 9, Eq. 10, Eq. 11, and Section 3.3 Eq. 12).  Only the tests, the
+smoke check and the benchmark's CPU-baseline leg may import it.  It shares no
+code with the CUDA path and never imports it.
+
+Everything is numpy float64.  The only library primitive used as a step is the
+matrix product for the logits (and for the two gradient contractions); rows are
+processed in chunks purely to bound memory -- rows are independent, so chunking
+changes nothing but the order in which dW's sum over rows is accumulated.
+
+Notation (Section 3.2): a draft block has K parallel positions k = 0..K-1; the
+rows of H are laid out block after block, row r = b*K + k.  y_r is the
+ground-truth token of row r.  c_k is the confidence in y at position k (Eq. 9),
+s_k the exclusive prefix product of confidences (Eq. 10), used as a
+stop-gradient weight on the per-token cross-entropy (Eq. 11).
+
+Readings taken where the paper is silent (each also listed in the design notes):
+  * confidence source: the paper's Eq. 9 uses the target model's probability of
+    the label.  Here the default is the probability the head itself (H, W)
+    assigns to the label; `conf_ext` supplies externally computed confidences
+    (the paper's target-model mode).  Either way the weight is a constant under
+    differentiation (sentence after Eq. 10: "stop-gradient weight").
+  * normalisation: Eq. 11 has 1/K for one block; over a batch with a valid-row
+    mask the loss is divided by N = number of valid rows (equals the mean over
+    blocks of Eq. 11 when all rows are valid; equals mean CE for unit weights,
+    Eq. 5).
+  * invalid rows (padding, rows past the sequence end in Eq. 12's n <= N-k):
+    weight 0, no loss, no gradient, and factor 1 in the prefix product.
+  * a label outside [0, V) on a valid row makes the row invalid.
+
+Pins (tests/test_oracle_pins.py): Eq. 5 degenerate case against
+torch.nn.functional.cross_entropy, K = 1, constant confidence = fixed decay
+gamma**k, W = 0 closed form, the Eq. 6/Eq. 8 acceptance-length identity, a hand
+example, finite differences with frozen weights, brute force in pure Python.
+Parity unpinned by the paper (fixed by the readings above): the confidence
+source, the batch normaliser, and the treatment of masked rows.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "effective_valid",
+    "softmax_stats",
+    "cat_weights",
+    "cat_weights_f32",
+    "cat_forward",
+    "cat_backward",
+    "cat_forward_backward",
+    "cat_dH_rows",
+    "cat_dW_rows",
+]
+
+
+def _as_f64(x) -> np.ndarray:
+    """Widen an array-like (numpy, or a torch CPU tensor incl. bf16) to float64 exactly."""
+    if hasattr(x, "detach"):  # torch tensor, without importing torch here
+        x = x.detach().to("cpu").double().numpy()
+    return np.ascontiguousarray(x, dtype=np.float64)
+
+
+def _as_i64(x) -> np.ndarray:
+    if hasattr(x, "detach"):
+        x = x.detach().to("cpu").numpy()
+    return np.ascontiguousarray(x, dtype=np.int64)
+
+
+def effective_valid(labels, valid, V: int) -> np.ndarray:
+    """Row r takes part iff its mask bit is set and 0 <= y_r < V (boolean array)."""
+    y = _as_i64(labels)
+    ok = (y >= 0) & (y < V)
+    if valid is not None:
+        v = valid.detach().to("cpu").numpy() if hasattr(valid, "detach") else np.asarray(valid)
+        ok &= v.astype(bool)
+    return ok
+
+
+def softmax_stats(z: np.ndarray):
+    """Row-wise m = max z, l = sum exp(z - m), lse = m + log l (the log-partition in Eq. 11's log P)."""
+    m = z.max(axis=1)
+    l = np.exp(z - m[:, None]).sum(axis=1)
+    return m, l, m + np.log(l)
+
+
+def cat_weights(conf: np.ndarray, eff_valid: np.ndarray, K: int) -> np.ndarray:
+    """Eq. 10: s_k = prod_{j<k} c_j, s_0 = 1, independently inside every block of K rows.
+
+    Invalid rows get weight 0 and contribute the factor 1 to the product.
+    Sequential in k (left to right), float64.
+    """
+    c = np.asarray(conf, dtype=np.float64).reshape(-1, K)
+    ok = np.asarray(eff_valid, dtype=bool).reshape(-1, K)
+    w = np.zeros_like(c)
+    s = np.ones(c.shape[0], dtype=np.float64)
+    for k in range(K):
+        w[:, k] = np.where(ok[:, k], s, 0.0)
+        s = np.where(ok[:, k], s * c[:, k], s)
+    return w.reshape(-1)
+
+
+def cat_weights_f32(conf_f32: np.ndarray, eff_valid: np.ndarray, K: int) -> np.ndarray:
+    """Eq. 10 in IEEE binary32, left to right, round-to-nearest-even, denormals kept.
+
+    Reference for the bit-exact weight check: given float32 confidences it
+    returns the float32 sequential product ((1*c_0)*c_1)*... per block.
+    """
+    c = np.asarray(conf_f32)
+    if c.dtype != np.float32:
+        raise TypeError("cat_weights_f32 wants float32 confidences")
+    c = c.reshape(-1, K)
+    ok = np.asarray(eff_valid, dtype=bool).reshape(-1, K)
+    w = np.zeros_like(c)
+    s = np.ones(c.shape[0], dtype=np.float32)
+    for k in range(K):
+        w[:, k] = np.where(ok[:, k], s, np.float32(0.0))
+        s = np.where(ok[:, k], (s * c[:, k]).astype(np.float32), s)
+    return w.reshape(-1)
+
+
+def cat_forward(H, W, labels, valid, K: int, conf_ext=None, row_chunk: int = 1024,
+                check_rows_sum_to_one: bool = True) -> dict:
+    """Forward pass of the CAT objective (Eq. 9-11) over T = B*K rows.
+
+    Returns a dict with float64 arrays lse[T], z_label[T], conf[T], weight[T],
+    row_ce[T] (= -log P(y_r), 0 on invalid rows), eff_valid[T] (bool),
+    n_valid (int) and the scalar loss = (1/N) sum_r w_r * row_ce_r.
+    """
+    Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
+    T, d = Hd.shape
+    V = Wd.shape[0]
+    if Wd.shape[1] != d or y.shape[0] != T or K < 1 or T % K != 0:
+        raise ValueError("bad shapes")
+    ok = effective_valid(y, valid, V)
+    ysafe = np.where(ok, y, 0)
+    lse = np.empty(T)
+    zy = np.empty(T)
+    for r0 in range(0, T, row_chunk):
+        r1 = min(T, r0 + row_chunk)
+        z = Hd[r0:r1] @ Wd.T                       # logits of these rows over the whole vocabulary
+        _, _, lse[r0:r1] = softmax_stats(z)
+        if check_rows_sum_to_one:
+            p_sum = np.exp(z - lse[r0:r1, None]).sum(axis=1)
+            assert np.all(np.abs(p_sum - 1.0) <= 1e-12), "softmax rows do not sum to 1"
+        zy[r0:r1] = z[np.arange(r1 - r0), ysafe[r0:r1]]
+    p_label = np.exp(zy - lse)                      # probability of the label token
+    if conf_ext is None:
+        conf = np.where(ok, p_label, 1.0)           # Eq. 9 evaluated with this head
+    else:
+        conf = np.where(ok, _as_f64(conf_ext), 1.0)  # Eq. 9 from the target model, supplied
+    w = cat_weights(conf, ok, K)                    # Eq. 10
+    row_ce = np.where(ok, lse - zy, 0.0)            # -log P(y_r)
+    n_valid = int(ok.sum())
+    loss = float((w * row_ce).sum() / n_valid) if n_valid > 0 else 0.0   # Eq. 11, batch mean
+    return dict(loss=loss, lse=lse, z_label=zy, conf=conf, weight=w, row_ce=row_ce,
+                eff_valid=ok, n_valid=n_valid)
+
+
+def cat_backward(H, W, labels, K: int, fwd: dict, g: float = 1.0, row_chunk: int = 1024):
+    """Gradients of g * loss w.r.t. H and W with the weights held constant (stop-gradient).
+
+    dz[r, v] = g * (w_r / N) * (p[r, v] - [v == y_r]);  dH = dz W;  dW = dz^T H.
+    """
+    Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
+    T, d = Hd.shape
+    V = Wd.shape[0]
+    ok, w, lse, N = fwd["eff_valid"], fwd["weight"], fwd["lse"], fwd["n_valid"]
+    dH = np.zeros((T, d))
+    dW = np.zeros((V, d))
+    if N == 0:
+        return dH, dW
+    coef = np.where(ok, g * w / N, 0.0)
+    ysafe = np.where(ok, y, 0)
+    for r0 in range(0, T, row_chunk):
+        r1 = min(T, r0 + row_chunk)
+        z = Hd[r0:r1] @ Wd.T
+        p = np.exp(z - lse[r0:r1, None])
+        p[np.arange(r1 - r0), ysafe[r0:r1]] -= 1.0
+        dz = p * coef[r0:r1, None]
+        dH[r0:r1] = dz @ Wd
+        dW += dz.T @ Hd[r0:r1]
+    return dH, dW
+
+
+def cat_forward_backward(H, W, labels, valid, K: int, conf_ext=None, g: float = 1.0,
+                         row_chunk: int = 1024):
+    fwd = cat_forward(H, W, labels, valid, K, conf_ext=conf_ext, row_chunk=row_chunk)
+    dH, dW = cat_backward(H, W, labels, K, fwd, g=g, row_chunk=row_chunk)
+    return fwd, dH, dW
+
+
+def cat_dH_rows(H, W, labels, fwd_rows: dict, rows: np.ndarray, n_valid_total: int, g: float = 1.0):
+    """dH for a chosen set of rows, given the forward state of exactly those rows.
+
+    `fwd_rows` holds lse / weight / eff_valid for `rows` (in that order);
+    `n_valid_total` is N of the whole batch.
+    """
+    Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
+    rows = np.asarray(rows, dtype=np.int64)
+    ok = fwd_rows["eff_valid"]
+    z = Hd[rows] @ Wd.T
+    p = np.exp(z - fwd_rows["lse"][:, None])
+    p[np.arange(len(rows)), np.where(ok, y[rows], 0)] -= 1.0
+    coef = np.where(ok, g * fwd_rows["weight"] / n_valid_total, 0.0)
+    return (p * coef[:, None]) @ Wd
+
+
+def cat_dW_rows(H, W, labels, fwd: dict, vocab_rows: np.ndarray, g: float = 1.0):
+    """dW[v, :] for chosen token ids v, given the forward state of ALL rows."""
+    Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
+    v = np.asarray(vocab_rows, dtype=np.int64)
+    ok, N = fwd["eff_valid"], fwd["n_valid"]
+    z = Hd @ Wd[v].T                                  # [T, len(v)]
+    p = np.exp(z - fwd["lse"][:, None])
+    p -= (y[:, None] == v[None, :]) & ok[:, None]
+    coef = np.where(ok, g * fwd["weight"] / N, 0.0)
+    return (p * coef[:, None]).T @ Hd

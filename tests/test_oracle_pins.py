@@ -1,0 +1,282 @@
+"""Pins for the fp64 oracle: it is checked against what the paper's formulas and plain
+mathematics fix, never against itself and never against the CUDA path.
+
+Each test names the equation it pins.  A dropped term, a wrong sign or index, an inclusive
+instead of exclusive product, a gradient through the weights, or a wrong normaliser fails
+at least one of them.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cat_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_problem(seed, T, d, V, scale=0.3, masked=False):
+    rng = np.random.default_rng(seed)
+    H = rng.standard_normal((T, d))
+    W = rng.standard_normal((V, d)) * scale
+    y = rng.integers(0, V, size=T)
+    valid = np.ones(T, dtype=np.uint8)
+    if masked:
+        valid[rng.random(T) < 0.25] = 0
+    return H, W, y, valid
+
+
+# ---------------------------------------------------------------- Eq. 10: hand examples
+def _read_hand_examples():
+    out = []
+    with open(os.path.join(GOLDEN, "eq10_hand_examples.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, c, v, w = [p.strip() for p in line.split("|")]
+            out.append((int(k), np.array(c.split(), float), np.array(v.split(), int), np.array(w.split(), float)))
+    return out
+
+
+@pytest.mark.parametrize("K,c,v,w", _read_hand_examples())
+def test_eq10_hand_examples(K, c, v, w):
+    assert np.array_equal(O.cat_weights(c, v.astype(bool), K), w)
+    assert np.array_equal(O.cat_weights_f32(c.astype(np.float32), v.astype(bool), K), w.astype(np.float32))
+
+
+def test_eq10_first_weight_is_one_and_recurrence():
+    rng = np.random.default_rng(1)
+    K, B = 16, 37
+    c = rng.random(B * K)
+    ok = np.ones(B * K, bool)
+    w = O.cat_weights(c, ok, K).reshape(B, K)
+    cc = c.reshape(B, K)
+    assert np.all(w[:, 0] == 1.0)                                   # s_0 := 1
+    assert np.allclose(w[:, 1:], w[:, :-1] * cc[:, :-1], rtol=0, atol=0)  # s_{k+1} = s_k c_k
+    assert np.all(np.diff(w, axis=1) <= 0) and np.all((w >= 0) & (w <= 1))
+    # the weight of row k must not contain c_k itself (exclusive product)
+    c2 = cc.copy(); c2[:, 5] = 0.123
+    w2 = O.cat_weights(c2.reshape(-1), ok, K).reshape(B, K)
+    assert np.array_equal(w2[:, :6], w[:, :6]) and not np.array_equal(w2[:, 6], w[:, 6])
+
+
+def test_eq6_eq8_acceptance_length_identity():
+    # sum_k s_k c_k == sum_k prod_{j<=k} c_j  (Eq. 6 rewritten as Eq. 8)
+    rng = np.random.default_rng(2)
+    K = 8
+    c = rng.random(5 * K)
+    w = O.cat_weights(c, np.ones_like(c, bool), K).reshape(5, K)
+    lhs = (w * c.reshape(5, K)).sum(axis=1)
+    rhs = np.cumprod(c.reshape(5, K), axis=1).sum(axis=1)
+    assert np.allclose(lhs, rhs, rtol=1e-14)
+
+
+def test_constant_confidence_is_fixed_decay():
+    # with c == gamma, Eq. 10 gives s_k = gamma^k: the fixed position decay the paper ablates against
+    H, W, y, valid = _rand_problem(3, 4 * 8, 8, 32)
+    for gamma in (1.0, 0.8, 0.6):
+        fwd = O.cat_forward(H, W, y, valid, 8, conf_ext=np.full(32, gamma))
+        expect = np.tile(gamma ** np.arange(8), 4)
+        assert np.allclose(fwd["weight"], expect, rtol=1e-14)
+        ce = fwd["lse"] - fwd["z_label"]
+        assert math.isclose(fwd["loss"], float((expect * ce).mean()), rel_tol=1e-13)
+
+
+# ---------------------------------------------------------------- Eq. 5 / Eq. 11 degenerate cases
+def _torch_ce(H, W, y, valid, reduction_n):
+    Ht = torch.tensor(H, dtype=torch.float64, requires_grad=True)
+    Wt = torch.tensor(W, dtype=torch.float64, requires_grad=True)
+    yt = torch.tensor(np.where(valid.astype(bool), y, -100))
+    loss = torch.nn.functional.cross_entropy(Ht @ Wt.T, yt, ignore_index=-100, reduction="sum") / reduction_n
+    loss.backward()
+    return loss.item(), Ht.grad.numpy(), Wt.grad.numpy()
+
+
+@pytest.mark.parametrize("masked", [False, True])
+def test_unit_confidence_reduces_to_mean_cross_entropy(masked):
+    # all prefix confidences 1 => s == 1 => Eq. 11 is the uniform PARD loss of Eq. 5
+    H, W, y, valid = _rand_problem(4, 6 * 4, 8, 32, masked=masked)
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, 4, conf_ext=np.ones(24), g=1.0)
+    n = int(valid.sum())
+    loss_t, dH_t, dW_t = _torch_ce(H, W, y, valid, n)
+    assert fwd["n_valid"] == n
+    assert np.array_equal(fwd["weight"], valid.astype(float))
+    assert math.isclose(fwd["loss"], loss_t, rel_tol=1e-12)
+    assert np.allclose(dH, dH_t, rtol=1e-10, atol=1e-14)
+    assert np.allclose(dW, dW_t, rtol=1e-10, atol=1e-14)
+
+
+def test_K1_is_plain_cross_entropy_in_self_confidence_mode():
+    # K = 1: every row is position 0, s_0 := 1 whatever the confidences are
+    H, W, y, valid = _rand_problem(5, 20, 8, 32, masked=True)
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, 1, g=0.7)
+    loss_t, dH_t, dW_t = _torch_ce(H, W, y, valid, int(valid.sum()))
+    assert math.isclose(fwd["loss"], loss_t, rel_tol=1e-12)
+    assert np.allclose(dH, 0.7 * dH_t, rtol=1e-10, atol=1e-14)
+    assert np.allclose(dW, 0.7 * dW_t, rtol=1e-10, atol=1e-14)
+
+
+def test_W_zero_closed_form():
+    # W = 0: p == 1/V, c = 1/V, s_k = V^-k, loss = (ln V / K) (1 - V^-K)/(1 - 1/V); dH = 0
+    T, d, V, K = 24, 8, 32, 4
+    H, _, y, valid = _rand_problem(6, T, d, V)
+    W = np.zeros((V, d))
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, K)
+    assert np.allclose(fwd["conf"], 1.0 / V, rtol=1e-14)
+    assert np.allclose(fwd["weight"].reshape(-1, K), (1.0 / V) ** np.arange(K), rtol=1e-13)
+    closed = math.log(V) / K * (1 - V ** (-K)) / (1 - 1 / V)
+    assert math.isclose(fwd["loss"], closed, rel_tol=1e-13)
+    assert np.all(dH == 0)
+    w = fwd["weight"]
+    expect_dW = np.zeros((V, d))
+    for r in range(T):
+        for v in range(V):
+            expect_dW[v] += (w[r] / T) * (1.0 / V - (1.0 if v == y[r] else 0.0)) * H[r]
+    assert np.allclose(dW, expect_dW, rtol=1e-12, atol=1e-16)
+
+
+# ---------------------------------------------------------------- brute force, pure Python
+def _brute_force(H, W, y, valid, K, g):
+    """Eq. 9-11 and the frozen-weight gradient in pure Python lists and math.exp, no max-subtraction."""
+    T, d, V = len(H), len(H[0]), len(W)
+    p = []
+    for r in range(T):
+        z = [sum(H[r][i] * W[v][i] for i in range(d)) for v in range(V)]
+        e = [math.exp(t) for t in z]
+        s = sum(e)
+        p.append([t / s for t in e])
+    ok = [bool(valid[r]) and 0 <= y[r] < V for r in range(T)]
+    N = sum(ok)
+    w = [0.0] * T
+    for b in range(T // K):
+        s = 1.0
+        for k in range(K):
+            r = b * K + k
+            if ok[r]:
+                w[r] = s
+                s *= p[r][y[r]]
+    loss = sum(-w[r] * math.log(p[r][y[r]]) for r in range(T) if ok[r]) / N
+    dH = [[0.0] * d for _ in range(T)]
+    dW = [[0.0] * d for _ in range(V)]
+    for r in range(T):
+        if not ok[r]:
+            continue
+        for v in range(V):
+            dz = g * w[r] / N * (p[r][v] - (1.0 if v == y[r] else 0.0))
+            for i in range(d):
+                dH[r][i] += dz * W[v][i]
+                dW[v][i] += dz * H[r][i]
+    return loss, w, dH, dW
+
+
+def test_brute_force_tiny_with_mask_and_bad_label():
+    T, d, V, K = 12, 4, 7, 4
+    H, W, y, valid = _rand_problem(7, T, d, V, scale=0.8, masked=True)
+    y = y.copy(); y[3] = V + 2; valid[3] = 1; valid[0] = 1; valid[1] = 1   # out-of-range label on a valid row
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, K, g=1.3)
+    loss_b, w_b, dH_b, dW_b = _brute_force(H.tolist(), W.tolist(), y.tolist(), valid.tolist(), K, 1.3)
+    assert math.isclose(fwd["loss"], loss_b, rel_tol=1e-12)
+    assert np.allclose(fwd["weight"], w_b, rtol=1e-12)
+    assert np.allclose(dH, dH_b, rtol=1e-10, atol=1e-15)
+    assert np.allclose(dW, dW_b, rtol=1e-10, atol=1e-15)
+    assert fwd["weight"][3] == 0 and np.all(dH[3] == 0)
+
+
+# ---------------------------------------------------------------- gradients: stop-gradient on s
+def _loss_with_weights(H, W, y, valid, K, w_fixed):
+    fwd = O.cat_forward(H, W, y, valid, K)
+    ce = fwd["lse"] - fwd["z_label"]
+    return float((w_fixed * np.where(fwd["eff_valid"], ce, 0.0)).sum() / fwd["n_valid"])
+
+
+def test_finite_differences_with_frozen_weights_and_converse():
+    T, d, V, K = 8, 8, 32, 4
+    H, W, y, valid = _rand_problem(8, T, d, V, scale=0.5)
+    H[:, :] += 2.0 * W[y]            # push confidences up so later positions carry weight
+    valid[5] = 0
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, K)
+    w0 = fwd["weight"]
+    assert w0.reshape(-1, K)[:, 1:].max() > 1e-2
+    eps = 1e-6
+    rng = np.random.default_rng(9)
+    worst = 0.0
+    moved = 0.0
+    for _ in range(40):
+        if rng.random() < 0.5:
+            r, i = rng.integers(T), rng.integers(d)
+            def bump(s, r=r, i=i):
+                Hp = H.copy(); Hp[r, i] += s; return Hp, W
+            ana = dH[r, i]
+        else:
+            v, i = rng.integers(V), rng.integers(d)
+            def bump(s, v=v, i=i):
+                Wp = W.copy(); Wp[v, i] += s; return H, Wp
+            ana = dW[v, i]
+        Hp, Wp = bump(eps); Hm, Wm = bump(-eps)
+        fd_frozen = (_loss_with_weights(Hp, Wp, y, valid, K, w0) - _loss_with_weights(Hm, Wm, y, valid, K, w0)) / (2 * eps)
+        fd_free = (O.cat_forward(Hp, Wp, y, valid, K)["loss"] - O.cat_forward(Hm, Wm, y, valid, K)["loss"]) / (2 * eps)
+        # central differences carry ~1e-10 absolute rounding noise (loss ~ 1, eps 1e-6)
+        worst = max(worst, abs(fd_frozen - ana) / (abs(ana) + 1e-3))
+        moved = max(moved, abs(fd_free - ana) / (abs(ana) + 1e-3))
+    assert worst <= 1e-7          # the analytic gradient treats s as a constant ...
+    assert moved >= 1e-2          # ... and differs from the derivative of the un-frozen loss
+
+
+# ---------------------------------------------------------------- invariants that hold at any size
+def test_invariants():
+    T, d, V, K = 64, 16, 50, 8
+    H, W, y, valid = _rand_problem(10, T, d, V, masked=True)
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, K, g=2.0)
+    ok = fwd["eff_valid"]
+    # sum_v dz[r, v] = 0  =>  dW summed over the vocabulary vanishes
+    assert np.allclose(dW.sum(axis=0), 0, atol=1e-15)
+    assert np.all(dH[~ok] == 0)
+    p = np.exp(H @ W.T - fwd["lse"][:, None])
+    assert np.allclose(p.sum(axis=1), 1.0, rtol=0, atol=1e-12)
+    coef = 2.0 * fwd["weight"] / fwd["n_valid"]
+    expect = coef[:, None] * (p @ W - W[np.where(ok, y, 0)])
+    assert np.allclose(dH[ok], expect[ok], rtol=1e-10, atol=1e-16)
+    rows = np.array([3, 17, 40])
+    sub = dict(lse=fwd["lse"][rows], weight=fwd["weight"][rows], eff_valid=ok[rows])
+    assert np.allclose(O.cat_dH_rows(H, W, y, sub, rows, fwd["n_valid"], g=2.0), dH[rows], rtol=1e-12, atol=1e-18)
+    vs = np.array([0, 7, 49, int(y[0])])
+    assert np.allclose(O.cat_dW_rows(H, W, y, fwd, vs, g=2.0), dW[vs], rtol=1e-12, atol=1e-18)
+
+
+def test_all_invalid_gives_zero():
+    H, W, y, _ = _rand_problem(11, 8, 4, 9)
+    fwd, dH, dW = O.cat_forward_backward(H, W, y, np.zeros(8, np.uint8), 4)
+    assert fwd["loss"] == 0.0 and fwd["n_valid"] == 0 and not dH.any() and not dW.any()
+
+
+def test_row_chunking_does_not_change_results():
+    H, W, y, valid = _rand_problem(12, 40, 8, 33, masked=True)
+    a = O.cat_forward_backward(H, W, y, valid, 4, row_chunk=1024)
+    b = O.cat_forward_backward(H, W, y, valid, 4, row_chunk=7)
+    assert math.isclose(a[0]["loss"], b[0]["loss"], rel_tol=1e-14)
+    assert np.allclose(a[1], b[1], rtol=1e-13, atol=1e-18) and np.allclose(a[2], b[2], rtol=1e-12, atol=1e-18)
+
+
+# ---------------------------------------------------------------- binary32 weight routine
+def test_weights_f32_is_sequential_binary32_with_denormals():
+    rng = np.random.default_rng(13)
+    K = 32
+    c = rng.random(3 * K).astype(np.float32) * np.float32(0.2)
+    ok = np.ones(3 * K, bool); ok[40] = False
+    w = O.cat_weights_f32(c, ok, K)
+    for b in range(3):
+        s = np.float32(1.0)
+        for k in range(K):
+            r = b * K + k
+            if ok[r]:
+                assert w[r].tobytes() == s.tobytes()
+                s = np.float32(s * c[r])
+            else:
+                assert w[r] == 0
+    # V^-k underflows gradually: denormal results are kept, not flushed
+    c = np.full(16, np.float32(2.0 ** -10), np.float32)
+    w = O.cat_weights_f32(c, np.ones(16, bool), 16)
+    assert w[14] == np.float32(2.0 ** -140) and w[14] != 0 and w[15] == 0
