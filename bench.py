@@ -1,0 +1,281 @@
+#!/usr/bin/env python
+"""Benchmark of the CAT loss hot path (fused LM head + CAT-weighted cross-entropy, fwd + bwd).
+
+One step = cat_loss_fwd + cat_loss_bwd over one synthetic draft-training batch of the
+Llama-3.2-1B-shaped head config (T=16384 rows in blocks of K=8, d=2048, V=128256, bf16).
+Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
+metric with host (pinned) buffers, host<->device copies inside the timed region; `roofline`
+is the forward logits GEMM (2*T*d*V flops per launch) against the measured dense bf16 peak;
+`cpu_baseline` is the fp64 oracle timed on this machine's host cores on a bounded sample.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+For N > 1 launch with torch.distributed.run; ranks run independent batches (draft blocks are
+independent, so the path shards by rows with no data-path collective: weak scaling).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+METRIC = "cat_loss_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(burst=float(j["bf16_tflops"]), sustained=float(j["bf16_tflops_sustained"]), hbm=float(j["hbm_gbs"]),
+                    source="measured")
+    return dict(burst=1590.0, sustained=1400.0, hbm=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.idx, self.rows, self.proc = device_index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.idx)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.25)
+        self.proc.terminate()
+        sm = [float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
+        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in self.rows:
+            if len(r) >= 9:
+                for n, v in zip(names, r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_sample_rate(batch, rows, steps=1):
+    """tokens/s of the fp64 oracle (fwd + bwd, incl. those rows' dW contribution) on the first `rows` rows."""
+    from oracle import cat_oracle as O
+    H, y, v = batch.H[:rows], batch.labels[:rows], batch.valid[:rows]
+    Hd, Wd = H.double().numpy(), batch.W.double().numpy()
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        O.cat_forward_backward(Hd, Wd, y, v, batch.K, row_chunk=256)
+        times.append(time.perf_counter() - t0)
+    return rows / (sum(times) / len(times)), sum(times) / len(times) * 1e3
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--rows", type=int, default=0, help="override T (debug / profiling of a small case)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2605_08632_b200 import synth
+    spec = synth.CONFIGS[args.config]
+    T = args.rows if args.rows else spec.T
+    cfg = dict(workload=f"config{args.config}:{spec.name}", T=T, K=spec.K, d=spec.d, V=spec.V, rows_per_gpu=T,
+               labels=spec.labels, l2="inputs larger than L2 (W alone is %.0f MB)" % (spec.V * spec.d * 2 / 1e6),
+               parallelism=f"rows sharded by whole draft blocks x{args.gpus}, no collective")
+    flops_per_token = 6.0 * spec.d * spec.V
+
+    # ------------------------------------------------------------------ reference arm: the oracle on host cores
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        batch = synth.make_batch(args.config, T=min(T, 2048))
+        rows = 256
+        for _ in range(max(0, min(args.warmup, 1))):
+            oracle_sample_rate(batch, rows)
+        rate, ms = oracle_sample_rate(batch, rows, steps=max(1, args.steps))
+        cores = host_threads()
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": cfg,
+            "cpu_baseline": {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{rows} rows (whole K-blocks) of the workload per step, fwd+bwd incl. their dW contribution"},
+            "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}))
+        return
+
+    # ------------------------------------------------------------------ our arm
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path for the product")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2605_08632_b200.api import CatLoss
+    from paper_2605_08632_b200 import binding as B
+
+    batch = synth.make_batch(args.config, T=T)
+    if world > 1:   # every rank its own rows: re-draw H and labels with a rank-dependent seed
+        g = torch.Generator().manual_seed(1000 + rank)
+        batch.H = torch.randn(T, spec.d, generator=g).to(batch.torch_dtype)
+        batch.labels = torch.randint(0, spec.V, (T,), generator=g)
+    H, W = batch.H.to(dev), batch.W.to(dev)
+    labels, valid = batch.labels.to(dev), batch.valid.to(dev)
+    cl = CatLoss(T, spec.d, spec.V, spec.K, dtype=batch.torch_dtype)
+
+    def step():
+        cl.forward(H, W, labels, valid)
+        cl.backward(H, W, labels, valid)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    stream = torch.cuda.current_stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fwd_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    ev0.record(stream)
+    for i in range(args.steps):
+        fwd_ev[i][0].record(stream)
+        cl.forward(H, W, labels, valid)
+        fwd_ev[i][1].record(stream)
+        cl.backward(H, W, labels, valid)
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = ev0.elapsed_time(ev1)
+    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b in fwd_ev)
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * T / (ms_per_step * 1e-3)
+    assert cl.fwd_stats().device_status == 0 and cl.bwd_status() == 0, "device reported a timed-out wait"
+
+    # ------------------------------------------------------------------ end to end with host buffers
+    e2e = None
+    if not args.no_e2e:
+        Hh, Wh = batch.H.pin_memory(), batch.W.pin_memory()
+        yh, vh = batch.labels.pin_memory(), batch.valid.pin_memory()
+        loss_h = torch.empty(1, dtype=torch.float32).pin_memory()
+        dH_h = torch.empty(T, spec.d, dtype=batch.torch_dtype).pin_memory()
+        dW_h = torch.empty(spec.V, spec.d, dtype=torch.float32).pin_memory()
+
+        def e2e_step():
+            H.copy_(Hh, non_blocking=True); W.copy_(Wh, non_blocking=True)
+            labels.copy_(yh, non_blocking=True); valid.copy_(vh, non_blocking=True)
+            cl.forward(H, W, labels, valid)
+            cl.backward(H, W, labels, valid)
+            loss_h.copy_(cl.loss, non_blocking=True); dH_h.copy_(cl.dH, non_blocking=True); dW_h.copy_(cl.dW, non_blocking=True)
+
+        e2e_steps = max(2, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        ev0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        ev1.record(stream)
+        barrier()
+        e_ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = sum(x.numel() * x.element_size() for x in (Hh, Wh, yh, vh))
+        d2h = sum(x.numel() * x.element_size() for x in (loss_h, dH_h, dW_h))
+        e2e = {"value": world * T / (e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    fwd_flops = 2.0 * T * spec.d * spec.V
+    achieved = fwd_flops / (fwd_ms * 1e-3) / 1e12
+    tflops = value * flops_per_token / 1e12 / world
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if spec.dtype == "bf16" else "f32", "data": "synthetic", "config": cfg,
+        "tflops_6TdV_per_gpu": tflops,
+        "frac_of_peak": {"measured_burst": tflops / peaks["burst"], "measured_sustained": tflops / peaks["sustained"],
+                         "nominal_2250": tflops / 2250.0, "peaks": peaks["source"]},
+        "fwd_ms": fwd_ms, "bwd_ms": ms_per_step - fwd_ms,
+        "roofline": {"bound": "tensor", "kernel": "tc::gemm_kernel<K-major,K-major,EpiFwd> (forward logits + online softmax)",
+                     "achieved": achieved, "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["sustained"],
+                     "peak_kind": f"{peaks['source']} sustained bf16 (kernel timed inside the step loop); burst {peaks['burst']}",
+                     "flops_per_launch": fwd_flops, "traffic": None},
+        "clocks": clocks, "e2e": e2e,
+        "gpu_launches": None,
+    }
+    # launches of our kernels per step, as the library itself counts them:
+    # fwd = GEMM + row kernel(s) + finalize; bwd = scale + 3 GEMMs per vocabulary slab
+    per_step = B.cat_loss_launch_count(cl.shape, 0) + B.cat_loss_launch_count(cl.shape, 1)
+    out["gpu_launches"] = per_step * args.steps
+    out["launches_per_step"] = per_step
+
+    if not args.no_cpu_baseline:
+        rows = 512
+        rate, ms = oracle_sample_rate(batch, rows)
+        out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                               "sample": f"first {rows} rows (whole K-blocks) of the workload, fwd+bwd incl. their dW contribution, {ms:.0f} ms"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,156 @@
+/*
+ * cat_loss.h -- C ABI of the fused LM-head + Confidence-Adaptive Token (CAT) weighted
+ * cross-entropy for NVIDIA B200 (sm_100a).
+ *
+ * The operation is the training objective of the PARD-2 parallel draft model
+ * (Section 3.2, Eq. 9-11; batch form Section 3.3, Eq. 12).  For T = B*K rows laid out
+ * draft block after draft block (row r = b*K + k, k = 0..K-1 the draft position):
+ *
+ *     z[r, v]  = sum_i H[r, i] * W[v, i]                     logits over the whole vocabulary
+ *     lse[r]   = log sum_v exp z[r, v]
+ *     conf[r]  = exp(z[r, y_r] - lse[r])                     confidence in the label  (Eq. 9, evaluated
+ *                                                            with this head; or supplied, see conf_ext)
+ *     weight[r]= prod_{j<k, row bK+j valid} conf[bK+j]       exclusive prefix product, 1 at k = 0 (Eq. 10)
+ *     loss     = (1/N) sum_{valid r} weight[r] * (lse[r] - z[r, y_r])      (Eq. 11; N = #valid rows)
+ *
+ * and, with the weights held constant (the sentence after Eq. 10: stop-gradient),
+ *
+ *     dz[r, v] = g * weight[r]/N * (exp(z[r,v] - lse[r]) - [v == y_r]),   dH = dz W,   dW = dz^T H.
+ *
+ * A row is valid iff valid[r] != 0 (or valid == NULL) and 0 <= labels[r] < V.  Invalid rows
+ * get weight 0, add nothing to the loss or to the gradients, and count as the factor 1 in
+ * the prefix product of their block.  The T x V logits are never stored.
+ *
+ * General conventions
+ *   - Every data pointer is a DEVICE pointer owned by the caller, valid on the current
+ *     device, unless a parameter says "host".  cat_shape is read on the host.
+ *   - Nothing is allocated or freed here and no state is kept between calls.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and the call returns without synchronising.
+ *   - Argument errors that the host can see return a negative cat_status before anything is
+ *     launched; CAT_ERR_CUDA (a failed CUDA call) may come back after part of the work was
+ *     enqueued.  Nothing throws.  Conditions only the device can see (a wait inside a kernel that ran
+ *     out of time) are written to cat_stats.device_status / the workspace status word;
+ *     kernels never trap.
+ *   - Layout: H is [T, d] row-major with row pitch ldH elements, W is [V, d] row-major with
+ *     row pitch ldW elements.  For CAT_BF16: d % 8 == 0, ldH % 8 == 0, ldW % 8 == 0 and
+ *     16-byte aligned base pointers (TMA rules).  For CAT_F32: 4-byte alignment only.
+ *   - T % K == 0, K >= 1.  T, V < 2^31; d <= 65536.
+ */
+#ifndef CAT_LOSS_H_
+#define CAT_LOSS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CAT_OK = 0,
+    CAT_ERR_NULL = -1,       /* a required pointer is NULL                                  */
+    CAT_ERR_SHAPE = -2,      /* T, d, V, K out of range, T % K != 0, pitch < d               */
+    CAT_ERR_DTYPE = -3,      /* unknown dtype code or unsupported combination                */
+    CAT_ERR_ALIGN = -4,      /* pointer or pitch alignment rule broken                       */
+    CAT_ERR_WORKSPACE = -5,  /* workspace NULL or smaller than cat_loss_workspace_bytes()    */
+    CAT_ERR_ARCH = -6,       /* current device is not compute capability 10.x                */
+    CAT_ERR_CUDA = -7,       /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+    CAT_ERR_TIMEOUT = -8     /* reported in device_status: a bounded wait in a kernel expired */
+} cat_status;
+
+typedef enum { CAT_BF16 = 0, CAT_F32 = 1 } cat_dtype;
+
+/* Problem description, read on the host. */
+typedef struct {
+    int64_t T;         /* rows = draft blocks * K                                   */
+    int64_t d;         /* hidden size (contraction length of the logits)             */
+    int64_t V;         /* vocabulary size                                            */
+    int32_t K;         /* draft positions per block                                  */
+    int32_t in_dtype;  /* cat_dtype of H, W and dH.  CAT_BF16: tensor-core path with
+                          fp32 accumulation.  CAT_F32: fp32 FFMA path, fp32 throughout */
+    int32_t dW_dtype;  /* cat_dtype of dW: CAT_F32 (default) or CAT_BF16 (bf16 inputs only) */
+    int32_t slab_mib;  /* cap, in MiB, on the backward pass's dz scratch slab; 0 = default
+                          (2048).  Smaller caps mean more, narrower vocabulary slabs.     */
+    int64_t ldH;       /* row pitch of H and dH in elements, >= d                     */
+    int64_t ldW;       /* row pitch of W and dW in elements, >= d                     */
+} cat_shape;
+
+/* Per-call statistics written by cat_loss_fwd (device memory, 32 bytes). */
+typedef struct {
+    int64_t n_valid;          /* N: rows that took part                                              */
+    int64_t n_bad_labels;     /* rows with valid[r] != 0 whose label is outside [0, V)                */
+    float   sum_weight;       /* sum_r weight[r]                                                      */
+    float   est_accept_len;   /* mean over blocks of sum_k weight*conf: the estimate of Eq. 8         */
+    int32_t device_status;    /* CAT_OK or CAT_ERR_TIMEOUT                                            */
+    int32_t reserved;
+} cat_stats;
+
+/*
+ * Bytes of scratch the given pass needs for this shape: pass 0 = cat_loss_fwd,
+ * pass 1 = cat_loss_bwd.  Returns 0 if the shape is invalid.  The scratch holds the
+ * per-(row, vocabulary split) softmax partials in the forward pass, and in the backward
+ * pass one bounded slab of dz (bf16: rows x a slice of the vocabulary, at most about
+ * 2 GiB) plus an fp32 dH accumulator when the vocabulary is processed in more than one
+ * slab.  It never grows with T*V.
+ */
+size_t cat_loss_workspace_bytes(const cat_shape* shape, int pass);
+
+/*
+ * Forward pass: Eq. 9, Eq. 10, Eq. 11 as written at the top of this file.
+ *   H, W      [T, d], [V, d] of shape->in_dtype                               (device, in)
+ *   labels    [T] int64 token ids y_r                                          (device, in)
+ *   valid     [T] uint8, nonzero = row takes part; NULL = all rows             (device, in)
+ *   conf_ext  [T] fp32 confidences computed elsewhere (the paper's target-model
+ *             confidences, Eq. 9); NULL = use this head's own probability       (device, in)
+ *   loss      [1] fp32                                                          (device, out)
+ *   lse       [T] fp32 log-sum-exp of each row's logits                         (device, out)
+ *   conf      [T] fp32 confidence used in the product (1 for invalid rows)      (device, out)
+ *   weight    [T] fp32 CAT weight, the binary32 left-to-right product of conf
+ *             inside each block (0 for invalid rows)                            (device, out)
+ *   stats     optional cat_stats                                                (device, out)
+ *   workspace at least cat_loss_workspace_bytes(shape, 0) bytes, 256-byte aligned (device, scratch)
+ * lse and weight are the only state the backward pass needs.
+ * Returns CAT_OK or a negative cat_status.
+ */
+int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W,
+                 const int64_t* labels, const uint8_t* valid, const float* conf_ext,
+                 float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward pass: gradients of g * loss with the weights as constants (stop-gradient,
+ * Section 3.2).  The logits are recomputed slice by slice of the vocabulary;
+ * dz = weight * (softmax - one-hot) feeds the dH and dW contractions.
+ *   lse, weight  [T] fp32 as written by cat_loss_fwd                            (device, in)
+ *   grad_loss    [1] fp32 upstream scalar g (e.g. the paper's beta of Eq. 12);
+ *                NULL = 1.0                                                      (device, in)
+ *   dH           [T, d] of in_dtype, pitch ldH; fully overwritten                (device, out)
+ *   dW           [V, d] of dW_dtype, pitch ldW; overwritten, or added to when
+ *                accumulate_dW != 0                                              (device, in/out)
+ *   workspace    at least cat_loss_workspace_bytes(shape, 1) bytes, 256-byte aligned
+ * After the call completes, the first int32 of the workspace holds CAT_OK or
+ * CAT_ERR_TIMEOUT (a bounded wait inside a kernel expired; outputs are then undefined).
+ * Returns CAT_OK or a negative cat_status.
+ */
+int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W,
+                 const int64_t* labels, const uint8_t* valid,
+                 const float* lse, const float* weight, const float* grad_loss,
+                 void* dH, void* dW, int accumulate_dW,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Number of kernels of this library that the given pass (0 = cat_loss_fwd, 1 = cat_loss_bwd)
+ * launches for this shape: the logits GEMM, the per-row kernels and the final reduction in
+ * the forward pass; one set-up kernel plus three GEMMs per vocabulary slab in the backward
+ * pass.  Host-only; returns 0 for an invalid shape.
+ */
+int cat_loss_launch_count(const cat_shape* shape, int pass);
+
+/* Static, NUL-terminated description of a cat_status value (host pointer, never freed). */
+const char* cat_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAT_LOSS_H_ */

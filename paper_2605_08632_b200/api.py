@@ -1,0 +1,52 @@
+"""Convenience layer over the binding: owns the device buffers of one problem shape.
+
+It allocates outputs and workspaces with torch once, then every call goes straight to the
+C entry points.  No arithmetic of the method happens here.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class CatLoss:
+    """Buffers and calls for one (T, d, V, K, dtype) problem on the current CUDA device."""
+
+    def __init__(self, T: int, d: int, V: int, K: int, dtype: torch.dtype = torch.bfloat16,
+                 dW_dtype: torch.dtype = torch.float32, slab_mib: int = 0, device: str = "cuda"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("CatLoss needs a CUDA device; there is no CPU path")
+        code = {torch.bfloat16: B.CAT_BF16, torch.float32: B.CAT_F32}
+        self.dtype, self.dW_dtype = dtype, dW_dtype
+        self.shape = B.make_shape(T, d, V, K, code[dtype], code[dW_dtype], slab_mib=slab_mib)
+        self.T, self.d, self.V, self.K = T, d, V, K
+        dev = torch.device(device)
+        nf, nb = B.cat_loss_workspace_bytes(self.shape, 0), B.cat_loss_workspace_bytes(self.shape, 1)
+        if nf == 0 or nb == 0:
+            raise ValueError("invalid shape for cat_loss")
+        self.ws_fwd = torch.empty(nf, dtype=torch.uint8, device=dev)
+        self.ws_bwd = torch.empty(nb, dtype=torch.uint8, device=dev)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.lse = torch.empty(T, dtype=torch.float32, device=dev)
+        self.conf = torch.empty(T, dtype=torch.float32, device=dev)
+        self.weight = torch.empty(T, dtype=torch.float32, device=dev)
+        self.stats = torch.zeros(32, dtype=torch.uint8, device=dev)
+        self.dH = torch.empty(T, d, dtype=dtype, device=dev)
+        self.dW = torch.empty(V, d, dtype=dW_dtype, device=dev)
+
+    def forward(self, H, W, labels, valid=None, conf_ext=None):
+        B.cat_loss_fwd(self.shape, H, W, labels, valid, conf_ext, self.loss, self.lse, self.conf, self.weight,
+                       self.stats, self.ws_fwd)
+        return self.loss
+
+    def backward(self, H, W, labels, valid=None, grad_loss=None, accumulate_dW=False):
+        B.cat_loss_bwd(self.shape, H, W, labels, valid, self.lse, self.weight, grad_loss, self.dH, self.dW,
+                       accumulate_dW, self.ws_bwd)
+        return self.dH, self.dW
+
+    def bwd_status(self) -> int:
+        return int(self.ws_bwd[:4].view(torch.int32).item())
+
+    def fwd_stats(self):
+        return B.read_stats(self.stats)

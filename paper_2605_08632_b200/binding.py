@@ -1,0 +1,107 @@
+"""ctypes binding of libcat_loss.so: argument marshalling only.
+
+Each function has the name and the arguments of its C entry point (include/cat_loss.h).
+torch is used for device memory and streams; every step of the path runs in the library's
+own kernels.  There is no fallback: if the library is missing or a call fails, this raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+CAT_BF16, CAT_F32 = 0, 1
+CAT_OK = 0
+
+
+class cat_shape(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int64), ("d", ctypes.c_int64), ("V", ctypes.c_int64), ("K", ctypes.c_int32),
+                ("in_dtype", ctypes.c_int32), ("dW_dtype", ctypes.c_int32), ("slab_mib", ctypes.c_int32),
+                ("ldH", ctypes.c_int64), ("ldW", ctypes.c_int64)]
+
+
+class cat_stats(ctypes.Structure):
+    _fields_ = [("n_valid", ctypes.c_int64), ("n_bad_labels", ctypes.c_int64), ("sum_weight", ctypes.c_float),
+                ("est_accept_len", ctypes.c_float), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class CatError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where} failed: {code} ({cat_status_string(code)})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the sources are newer) the shared library; raises if that is impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = ctypes.CDLL(path)
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        L.cat_status_string.restype = ctypes.c_char_p
+        L.cat_status_string.argtypes = [ctypes.c_int]
+        L.cat_loss_workspace_bytes.restype = sz
+        L.cat_loss_workspace_bytes.argtypes = [ctypes.POINTER(cat_shape), ctypes.c_int]
+        L.cat_loss_launch_count.restype = ctypes.c_int
+        L.cat_loss_launch_count.argtypes = [ctypes.POINTER(cat_shape), ctypes.c_int]
+        L.cat_loss_fwd.restype = ctypes.c_int
+        L.cat_loss_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 10 + [vp, sz, vp]
+        L.cat_loss_bwd.restype = ctypes.c_int
+        L.cat_loss_bwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 9 + [ctypes.c_int, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def cat_status_string(code: int) -> str:
+    return lib().cat_status_string(int(code)).decode()
+
+
+def make_shape(T, d, V, K, in_dtype, dW_dtype=CAT_F32, ldH=None, ldW=None, slab_mib=0) -> cat_shape:
+    return cat_shape(T, d, V, K, in_dtype, dW_dtype, slab_mib, d if ldH is None else ldH, d if ldW is None else ldW)
+
+
+def cat_loss_workspace_bytes(shape: cat_shape, which: int) -> int:
+    return int(lib().cat_loss_workspace_bytes(ctypes.byref(shape), int(which)))
+
+
+def cat_loss_launch_count(shape: cat_shape, which: int) -> int:
+    return int(lib().cat_loss_launch_count(ctypes.byref(shape), int(which)))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, workspace) -> None:
+    """All tensor arguments are CUDA tensors (or None where the C API allows NULL); outputs are written in place."""
+    rc = lib().cat_loss_fwd(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(conf_ext),
+                            _ptr(loss), _ptr(lse), _ptr(conf), _ptr(weight), _ptr(stats),
+                            _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                            _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_loss_fwd")
+
+
+def cat_loss_bwd(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace) -> None:
+    rc = lib().cat_loss_bwd(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(lse), _ptr(weight),
+                            _ptr(grad_loss), _ptr(dH), _ptr(dW), int(bool(accumulate_dW)),
+                            _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                            _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_loss_bwd")
+
+
+def read_stats(stats_tensor: torch.Tensor) -> cat_stats:
+    """Copy a 32-byte device cat_stats (a uint8[32] tensor) to the host."""
+    raw = bytes(stats_tensor.cpu().numpy().tobytes())
+    return cat_stats.from_buffer_copy(raw)

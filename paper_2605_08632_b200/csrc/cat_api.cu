@@ -1,0 +1,423 @@
+// C ABI of the CAT loss library: host-side validation, workspace planning, tensor-map
+// construction and kernel launches.  Nothing here allocates device memory.
+#include "../../include/cat_loss.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "rowops.cuh"
+#include "simt.cuh"
+#include "tc_gemm.cuh"
+
+namespace {
+
+using namespace cat;
+
+constexpr int kPlanSMs = 148;            // B200: the static schedules are planned for 148 SMs
+constexpr size_t kHeaderBytes = 256;     // workspace header: int32 status at byte 0, fp32 g/N at byte 64
+constexpr size_t kScaleOffset = 64;
+constexpr int kMaxSplits = 128;
+constexpr long long kDefaultSlabMiB = 2048;
+
+inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+inline long long cdiv(long long a, long long b) { return (a + b - 1) / b; }
+
+// ------------------------------------------------------------------------------ validation
+int check_shape(const cat_shape* s) {
+    if (!s) return CAT_ERR_NULL;
+    if (s->T <= 0 || s->d <= 0 || s->V <= 0 || s->K < 1) return CAT_ERR_SHAPE;
+    if (s->T >= (1ll << 31) || s->V >= (1ll << 31) || s->d > 65536) return CAT_ERR_SHAPE;
+    if (s->T % s->K != 0) return CAT_ERR_SHAPE;
+    if (s->ldH < s->d || s->ldW < s->d) return CAT_ERR_SHAPE;
+    if (s->slab_mib < 0) return CAT_ERR_SHAPE;
+    if (s->in_dtype != CAT_BF16 && s->in_dtype != CAT_F32) return CAT_ERR_DTYPE;
+    if (s->dW_dtype != CAT_BF16 && s->dW_dtype != CAT_F32) return CAT_ERR_DTYPE;
+    if (s->in_dtype == CAT_F32 && s->dW_dtype != CAT_F32) return CAT_ERR_DTYPE;
+    if (s->in_dtype == CAT_BF16 && (s->d % 8 != 0 || s->ldH % 8 != 0 || s->ldW % 8 != 0)) return CAT_ERR_ALIGN;
+    return CAT_OK;
+}
+
+inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
+// ------------------------------------------------------------------------------ planning
+struct FwdPlan {
+    int S;                 // vocabulary splits
+    int n_row_ctas;        // CTAs of the per-row kernel (or of the per-block kernel for general K)
+    bool warp_scan;        // K is a power of two <= 32
+    size_t off_part_m, off_part_l, off_z_label, off_row_ce, off_partials, total;
+};
+
+FwdPlan plan_fwd(const cat_shape* s) {
+    FwdPlan p;
+    if (s->in_dtype == CAT_BF16) {
+        const long long num_m = cdiv(s->T, tc::BM), num_n = cdiv(s->V, tc::BN);
+        const long long smax = num_n < kMaxSplits ? num_n : kMaxSplits;
+        double best = 1e300;
+        p.S = 1;
+        for (long long S = 1; S <= smax; ++S) {
+            // persistent CTAs take items round-robin: waves * longest item, plus a small charge per split
+            const double cost = static_cast<double>(cdiv(num_m * S, kPlanSMs)) * static_cast<double>(cdiv(num_n, S)) + 1e-3 * S;
+            if (cost < best) { best = cost; p.S = static_cast<int>(S); }
+        }
+    } else {
+        const long long num_m = cdiv(s->T, simt::TM), num_n = cdiv(s->V, simt::TN);
+        long long S = (2 * kPlanSMs) / num_m;
+        if (S < 1) S = 1;
+        if (S > num_n) S = num_n;
+        if (S > 64) S = 64;
+        p.S = static_cast<int>(S);
+    }
+    p.warp_scan = s->K <= 32 && (s->K & (s->K - 1)) == 0;
+    const long long units = p.warp_scan ? s->T : s->T / s->K;
+    p.n_row_ctas = static_cast<int>(cdiv(units, rows::ROW_THREADS));
+    size_t off = kHeaderBytes;
+    p.off_part_m = off;  off = align256(off + sizeof(float) * p.S * s->T);
+    p.off_part_l = off;  off = align256(off + sizeof(float) * p.S * s->T);
+    p.off_z_label = off; off = align256(off + sizeof(float) * s->T);
+    p.off_row_ce = off;  off = align256(off + sizeof(float) * s->T);
+    p.off_partials = off; off = align256(off + sizeof(rows::CtaPartial) * p.n_row_ctas);
+    p.total = off;
+    return p;
+}
+
+struct BwdPlan {
+    long long Vs;          // slab width in vocabulary entries (multiple of 256)
+    int n_slabs;
+    size_t off_dz, off_dh_acc, total;
+};
+
+BwdPlan plan_bwd(const cat_shape* s) {
+    BwdPlan p;
+    const size_t elt = s->in_dtype == CAT_BF16 ? 2 : 4;
+    const long long mib = s->slab_mib > 0 ? s->slab_mib : kDefaultSlabMiB;
+    const long long v_pad = cdiv(s->V, 256) * 256;
+    long long Vs = (mib << 20) / static_cast<long long>(elt * s->T);
+    Vs = (Vs / 256) * 256;
+    if (Vs < 256) Vs = 256;
+    if (Vs > v_pad) Vs = v_pad;
+    p.n_slabs = static_cast<int>(cdiv(s->V, Vs));
+    p.Vs = cdiv(cdiv(s->V, p.n_slabs), 256) * 256;      // rebalance the slabs
+    p.n_slabs = static_cast<int>(cdiv(s->V, p.Vs));
+    size_t off = kHeaderBytes;
+    p.off_dz = off; off = align256(off + elt * static_cast<size_t>(s->T) * p.Vs);
+    p.off_dh_acc = off;
+    if (s->in_dtype == CAT_BF16 && p.n_slabs > 1) off = align256(off + sizeof(float) * static_cast<size_t>(s->T) * s->d);
+    p.total = off;
+    return p;
+}
+
+// ------------------------------------------------------------------------------ device / driver
+int check_device(int* sm_count) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_ARCH; }
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_ARCH; }
+    if (major != 10) return CAT_ERR_ARCH;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    *sm_count = sms;
+    return CAT_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major tensor [rows][cols] with row pitch `ld` elements, 128-byte swizzle.
+// box = {box_cols (inner, 64 elements = 128 bytes), box_rows}.  Out-of-range elements read as zero.
+int make_tmap(CUtensorMap* m, const void* base, long long rows, long long cols, long long ld, int box_cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return CAT_ERR_CUDA;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CAT_OK : CAT_ERR_CUDA;
+}
+inline int tmap_k_major(CUtensorMap* m, const void* base, long long mn, long long k, long long ld, int box_mn) {
+    return make_tmap(m, base, mn, k, ld, tc::BK, box_mn);          // [MN rows][K cols]
+}
+inline int tmap_mn_major(CUtensorMap* m, const void* base, long long k, long long mn, long long ld) {
+    return make_tmap(m, base, k, mn, ld, 64, tc::BK);              // [K rows][MN cols]
+}
+
+int band_tiles(long long d) {
+    long long b = (64ll << 20) / (tc::BM * d * 2);
+    return static_cast<int>(b < 1 ? 1 : b);
+}
+
+template <int A_MN, int B_MN, class Epi>
+int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& sched, const typename Epi::Params& ep,
+              int* status, int sm_count, cudaStream_t st) {
+    auto kern = tc::gemm_kernel<A_MN, B_MN, Epi>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) {
+        cudaGetLastError();
+        return CAT_ERR_CUDA;
+    }
+    const int grid = sched.n_items < sm_count ? sched.n_items : sm_count;
+    kern<<<grid, tc::NUM_THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, sched, ep, status);
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+}
+
+tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int band_m, int n_fastest) {
+    tc::Sched s;
+    s.num_m_tiles = static_cast<int>(cdiv(M, tc::BM));
+    s.num_n_tiles = static_cast<int>(cdiv(N, tc::BN));
+    s.num_kb = static_cast<int>(cdiv(Kd, tc::BK));
+    s.n_groups = n_groups > 0 ? n_groups : s.num_n_tiles;
+    s.band_m = band_m < 1 ? 1 : band_m;
+    s.n_fastest = n_fastest;
+    s.n_items = s.num_m_tiles * s.n_groups;
+    return s;
+}
+
+}  // namespace
+
+// =================================================================================== exports
+extern "C" {
+
+const char* cat_status_string(int status) {
+    switch (status) {
+        case CAT_OK: return "ok";
+        case CAT_ERR_NULL: return "a required pointer is NULL";
+        case CAT_ERR_SHAPE: return "invalid shape (T, d, V, K, pitches, T % K)";
+        case CAT_ERR_DTYPE: return "unsupported dtype combination";
+        case CAT_ERR_ALIGN: return "pointer or pitch alignment rule broken";
+        case CAT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CAT_ERR_ARCH: return "current device is not compute capability 10.x";
+        case CAT_ERR_CUDA: return "a CUDA call failed";
+        case CAT_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+        default: return "unknown status";
+    }
+}
+
+size_t cat_loss_workspace_bytes(const cat_shape* shape, int pass) {
+    if (check_shape(shape) != CAT_OK) return 0;
+    if (pass == 0) return plan_fwd(shape).total;
+    if (pass == 1) return plan_bwd(shape).total;
+    return 0;
+}
+
+int cat_loss_launch_count(const cat_shape* shape, int pass) {
+    if (check_shape(shape) != CAT_OK) return 0;
+    if (pass == 0) return 1 + (plan_fwd(shape).warp_scan ? 1 : 2) + 1;
+    if (pass == 1) return 1 + 3 * plan_bwd(shape).n_slabs;
+    return 0;
+}
+
+int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                 const float* conf_ext, float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!shape || !H || !W || !labels || !loss || !lse || !conf || !weight) return CAT_ERR_NULL;
+    const int sc = check_shape(shape);
+    if (sc != CAT_OK) return sc;
+    const bool bf16 = shape->in_dtype == CAT_BF16;
+    if (misaligned(H, bf16 ? 16 : 4) || misaligned(W, bf16 ? 16 : 4) || misaligned(labels, 8) || misaligned(loss, 4) ||
+        misaligned(lse, 4) || misaligned(conf, 4) || misaligned(weight, 4) || (conf_ext && misaligned(conf_ext, 4)) ||
+        (stats && misaligned(stats, 8)))
+        return CAT_ERR_ALIGN;
+    const FwdPlan plan = plan_fwd(shape);
+    if (!workspace || misaligned(workspace, 256) || workspace_bytes < plan.total) return CAT_ERR_WORKSPACE;
+    int sm_count = 0;
+    const int dc = check_device(&sm_count);
+    if (dc != CAT_OK) return dc;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws);
+    float* part_m = reinterpret_cast<float*>(ws + plan.off_part_m);
+    float* part_l = reinterpret_cast<float*>(ws + plan.off_part_l);
+    float* z_label = reinterpret_cast<float*>(ws + plan.off_z_label);
+    float* row_ce = reinterpret_cast<float*>(ws + plan.off_row_ce);
+    rows::CtaPartial* partials = reinterpret_cast<rows::CtaPartial*>(ws + plan.off_partials);
+    const int T = static_cast<int>(shape->T), V = static_cast<int>(shape->V);
+
+    CUtensorMap tmH, tmW;
+    if (bf16) {
+        if (tmap_k_major(&tmH, H, shape->T, shape->d, shape->ldH, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_k_major(&tmW, W, shape->V, shape->d, shape->ldW, tc::BN) != CAT_OK) return CAT_ERR_CUDA;
+    }
+    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+
+    if (bf16) {
+        const tc::Sched sched = make_sched(shape->T, shape->V, shape->d, plan.S, band_tiles(shape->d), 0);
+        tc::EpiFwd::Params ep;
+        ep.labels = reinterpret_cast<const long long*>(labels);
+        ep.part_m = part_m; ep.part_l = part_l; ep.z_label = z_label; ep.T = T; ep.V = V;
+        const int rc = launch_tc<0, 0, tc::EpiFwd>(tmH, tmW, sched, ep, status, sm_count, st);
+        if (rc != CAT_OK) return rc;
+    } else {
+        simt::Operands op;
+        op.A = static_cast<const float*>(H); op.sAm = shape->ldH; op.sAk = 1;
+        op.B = static_cast<const float*>(W); op.sBk = 1; op.sBn = shape->ldW;
+        op.M = T; op.N = V; op.Kd = static_cast<int>(shape->d); op.n_groups = plan.S;
+        simt::EpiParams ep;
+        memset(&ep, 0, sizeof(ep));
+        ep.labels = reinterpret_cast<const long long*>(labels);
+        ep.part_m = part_m; ep.part_l = part_l; ep.z_label = z_label; ep.V = V; ep.v0 = 0;
+        const dim3 grid(static_cast<unsigned>(cdiv(T, simt::TM)), static_cast<unsigned>(plan.S));
+        simt::gemm_kernel<simt::MODE_FWD><<<grid, simt::THREADS, 0, st>>>(op, ep);
+        if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+    }
+
+    rows::RowParams rp;
+    rp.part_m = part_m; rp.part_l = part_l; rp.z_label = z_label;
+    rp.labels = reinterpret_cast<const long long*>(labels); rp.valid = valid; rp.conf_ext = conf_ext;
+    rp.lse = lse; rp.conf = conf; rp.weight = weight; rp.row_ce = row_ce; rp.partials = partials;
+    rp.T = T; rp.V = V; rp.K = shape->K; rp.S = plan.S;
+    if (plan.warp_scan) {
+        rows::row_kernel<true><<<plan.n_row_ctas, rows::ROW_THREADS, 0, st>>>(rp);
+    } else {
+        rows::row_kernel<false><<<static_cast<unsigned>(cdiv(T, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(rp);
+        rows::block_scan_kernel<<<plan.n_row_ctas, rows::ROW_THREADS, 0, st>>>(rp);
+    }
+    rows::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(partials, plan.n_row_ctas, T / shape->K, loss,
+                                                         reinterpret_cast<rows::StatsOut*>(stats), status);
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+}
+
+int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                 const float* lse, const float* weight, const float* grad_loss, void* dH, void* dW, int accumulate_dW,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!shape || !H || !W || !labels || !lse || !weight || !dH || !dW) return CAT_ERR_NULL;
+    const int sc = check_shape(shape);
+    if (sc != CAT_OK) return sc;
+    const bool bf16 = shape->in_dtype == CAT_BF16;
+    const size_t in_al = bf16 ? 16 : 4;
+    if (misaligned(H, in_al) || misaligned(W, in_al) || misaligned(dH, in_al) || misaligned(dW, 16) || misaligned(labels, 8) ||
+        misaligned(lse, 4) || misaligned(weight, 4) || (grad_loss && misaligned(grad_loss, 4)))
+        return CAT_ERR_ALIGN;
+    const BwdPlan plan = plan_bwd(shape);
+    if (!workspace || misaligned(workspace, 256) || workspace_bytes < plan.total) return CAT_ERR_WORKSPACE;
+    int sm_count = 0;
+    const int dc = check_device(&sm_count);
+    if (dc != CAT_OK) return dc;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws);
+    float* scale = reinterpret_cast<float*>(ws + kScaleOffset);
+    const int T = static_cast<int>(shape->T), V = static_cast<int>(shape->V), d = static_cast<int>(shape->d);
+    const long long* y = reinterpret_cast<const long long*>(labels);
+
+    // tensor maps that do not depend on the slab
+    CUtensorMap tmH_k, tmH_mn;
+    if (bf16) {
+        if (tmap_k_major(&tmH_k, H, shape->T, shape->d, shape->ldH, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_mn_major(&tmH_mn, H, shape->T, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
+    }
+    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    rows::bwd_scale_kernel<<<1, 1024, 0, st>>>(y, valid, T, V, grad_loss, scale);
+    if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+
+    for (int sl = 0; sl < plan.n_slabs; ++sl) {
+        const long long v0 = static_cast<long long>(sl) * plan.Vs;
+        const long long width = (shape->V - v0) < plan.Vs ? (shape->V - v0) : plan.Vs;
+        const bool first = sl == 0, last = sl == plan.n_slabs - 1;
+        if (bf16) {
+            const __nv_bfloat16* Wb = static_cast<const __nv_bfloat16*>(W) + v0 * shape->ldW;
+            __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_dz);
+            float* dh_acc = reinterpret_cast<float*>(ws + plan.off_dh_acc);
+            CUtensorMap tmW_k, tmW_mn, tmDz_k, tmDz_mn;
+            if (tmap_k_major(&tmW_k, Wb, width, shape->d, shape->ldW, tc::BN) != CAT_OK) return CAT_ERR_CUDA;
+            if (tmap_mn_major(&tmW_mn, Wb, width, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
+            if (tmap_k_major(&tmDz_k, dz, shape->T, width, plan.Vs, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+            if (tmap_mn_major(&tmDz_mn, dz, shape->T, width, plan.Vs) != CAT_OK) return CAT_ERR_CUDA;
+            {   // recompute the logits of this slab and turn them into dz
+                const tc::Sched sched = make_sched(shape->T, width, shape->d, 0, band_tiles(shape->d), 0);
+                tc::EpiDz::Params ep;
+                ep.labels = y; ep.valid = valid; ep.lse = lse; ep.weight = weight; ep.dz = dz; ep.ld = plan.Vs;
+                ep.T = T; ep.V = V; ep.v0 = static_cast<int>(v0);
+                const int rc = launch_tc<0, 0, tc::EpiDz>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+                if (rc != CAT_OK) return rc;
+            }
+            {   // dW[v0 : v0 + width, :] = (g/N) dz^T H
+                const tc::Sched sched = make_sched(width, shape->d, shape->T, 0, 1, 1);
+                tc::EpiOut::Params ep;
+                memset(&ep, 0, sizeof(ep));
+                ep.alpha = scale; ep.M = static_cast<int>(width); ep.N = d; ep.ld_add = shape->ldW; ep.ld_out = shape->ldW;
+                if (shape->dW_dtype == CAT_F32) {
+                    ep.out_f32 = static_cast<float*>(dW) + v0 * shape->ldW;
+                    if (accumulate_dW) ep.add_f32 = ep.out_f32;
+                } else {
+                    ep.out_bf16 = static_cast<__nv_bfloat16*>(dW) + v0 * shape->ldW;
+                    if (accumulate_dW) ep.add_bf16 = ep.out_bf16;
+                }
+                const int rc = launch_tc<1, 1, tc::EpiOut>(tmDz_mn, tmH_mn, sched, ep, status, sm_count, st);
+                if (rc != CAT_OK) return rc;
+            }
+            {   // dH (+)= (g/N) dz W[v0 : v0 + width, :]
+                const tc::Sched sched = make_sched(shape->T, shape->d, width, 0, 1, 1);
+                tc::EpiOut::Params ep;
+                memset(&ep, 0, sizeof(ep));
+                ep.alpha = scale; ep.M = T; ep.N = d;
+                if (!first) { ep.add_f32 = dh_acc; ep.ld_add = shape->d; }
+                if (last) { ep.out_bf16 = static_cast<__nv_bfloat16*>(dH); ep.ld_out = shape->ldH; }
+                else { ep.out_f32 = dh_acc; ep.ld_out = shape->d; }
+                const int rc = launch_tc<0, 1, tc::EpiOut>(tmDz_k, tmW_mn, sched, ep, status, sm_count, st);
+                if (rc != CAT_OK) return rc;
+            }
+        } else {
+            const float* Hf = static_cast<const float*>(H);
+            const float* Wf = static_cast<const float*>(W) + v0 * shape->ldW;
+            float* dz = reinterpret_cast<float*>(ws + plan.off_dz);
+            const int w = static_cast<int>(width);
+            {
+                simt::Operands op;
+                op.A = Hf; op.sAm = shape->ldH; op.sAk = 1; op.B = Wf; op.sBk = 1; op.sBn = shape->ldW;
+                op.M = T; op.N = w; op.Kd = d; op.n_groups = static_cast<int>(cdiv(w, simt::TN));
+                simt::EpiParams ep;
+                memset(&ep, 0, sizeof(ep));
+                ep.labels = y; ep.valid = valid; ep.lse = lse; ep.weight = weight; ep.dz = dz; ep.ld_dz = plan.Vs;
+                ep.V = V; ep.v0 = static_cast<int>(v0);
+                const dim3 grid(static_cast<unsigned>(cdiv(T, simt::TM)), static_cast<unsigned>(op.n_groups));
+                simt::gemm_kernel<simt::MODE_DZ><<<grid, simt::THREADS, 0, st>>>(op, ep);
+            }
+            {   // dW slice = (g/N) dz^T H : A(m = v, k = r) = dz[r][v], B(k = r, n = i) = H[r][i]
+                simt::Operands op;
+                op.A = dz; op.sAm = 1; op.sAk = plan.Vs; op.B = Hf; op.sBk = shape->ldH; op.sBn = 1;
+                op.M = w; op.N = d; op.Kd = T; op.n_groups = static_cast<int>(cdiv(d, simt::TN));
+                simt::EpiParams ep;
+                memset(&ep, 0, sizeof(ep));
+                ep.alpha = scale; ep.out = static_cast<float*>(dW) + v0 * shape->ldW; ep.ld_out = shape->ldW;
+                if (accumulate_dW) { ep.add = ep.out; ep.ld_add = shape->ldW; }
+                const dim3 grid(static_cast<unsigned>(cdiv(w, simt::TM)), static_cast<unsigned>(op.n_groups));
+                simt::gemm_kernel<simt::MODE_OUT><<<grid, simt::THREADS, 0, st>>>(op, ep);
+            }
+            {   // dH (+)= (g/N) dz W slice : A(m = r, k = v) = dz[r][v], B(k = v, n = i) = W[v][i]
+                simt::Operands op;
+                op.A = dz; op.sAm = plan.Vs; op.sAk = 1; op.B = Wf; op.sBk = shape->ldW; op.sBn = 1;
+                op.M = T; op.N = d; op.Kd = w; op.n_groups = static_cast<int>(cdiv(d, simt::TN));
+                simt::EpiParams ep;
+                memset(&ep, 0, sizeof(ep));
+                ep.alpha = scale; ep.out = static_cast<float*>(dH); ep.ld_out = shape->ldH;
+                if (!first) { ep.add = ep.out; ep.ld_add = shape->ldH; }
+                const dim3 grid(static_cast<unsigned>(cdiv(T, simt::TM)), static_cast<unsigned>(op.n_groups));
+                simt::gemm_kernel<simt::MODE_OUT><<<grid, simt::THREADS, 0, st>>>(op, ep);
+            }
+            if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+        }
+    }
+    return CAT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,203 @@
+// Per-row kernels of the CAT loss: merging the vocabulary-split softmax partials into lse,
+// the confidence of Eq. 9, the segmented exclusive product scan of Eq. 10 (warp shuffles,
+// strictly left to right so the binary32 result equals the sequential product), the weighted
+// loss of Eq. 11 with a fixed-order reduction, and the small set-up kernel of the backward pass.
+// These touch O(T) data and are bandwidth/latency-bound; no tensor cores are involved.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cat {
+namespace rows {
+
+constexpr int ROW_THREADS = 256;
+
+// Per-CTA partial sums, reduced in a fixed order by finalize_kernel.
+struct CtaPartial {
+    double loss;        // sum_r weight_r * (lse_r - z[r, y_r])
+    double sum_w;       // sum_r weight_r
+    double sum_wc;      // sum_r weight_r * conf_r   (Eq. 8 estimate, summed over blocks)
+    long long n_valid;
+    long long n_bad;
+};
+
+struct RowParams {
+    const float* part_m;       // [S][T]
+    const float* part_l;       // [S][T]
+    const float* z_label;      // [T]
+    const long long* labels;   // [T]
+    const unsigned char* valid;  // [T] or nullptr
+    const float* conf_ext;     // [T] or nullptr
+    float* lse;                // [T]
+    float* conf;               // [T]
+    float* weight;             // [T]
+    float* row_ce;             // [T] scratch: lse - z_label (0 for invalid rows); used by the general-K path
+    CtaPartial* partials;      // [gridDim.x]
+    int T, V, K, S;
+};
+
+__device__ __forceinline__ void block_reduce_store(double loss, double sw, double swc, long long nv, long long nb,
+                                                   CtaPartial* out) {
+    // fixed-order tree: shuffles inside each warp, then warp 0 adds the per-warp sums in order
+    __shared__ double s_loss[ROW_THREADS / 32], s_sw[ROW_THREADS / 32], s_swc[ROW_THREADS / 32];
+    __shared__ long long s_nv[ROW_THREADS / 32], s_nb[ROW_THREADS / 32];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        loss += __shfl_down_sync(0xffffffffu, loss, off);
+        sw += __shfl_down_sync(0xffffffffu, sw, off);
+        swc += __shfl_down_sync(0xffffffffu, swc, off);
+        nv += __shfl_down_sync(0xffffffffu, nv, off);
+        nb += __shfl_down_sync(0xffffffffu, nb, off);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_loss[warp] = loss; s_sw[warp] = sw; s_swc[warp] = swc; s_nv[warp] = nv; s_nb[warp] = nb; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        CtaPartial p = {0.0, 0.0, 0.0, 0, 0};
+        for (int w = 0; w < ROW_THREADS / 32; ++w) {
+            p.loss += s_loss[w]; p.sum_w += s_sw[w]; p.sum_wc += s_swc[w]; p.n_valid += s_nv[w]; p.n_bad += s_nb[w];
+        }
+        *out = p;
+    }
+}
+
+// One thread per row.  SCAN = true: K is a power of two <= 32, the K rows of a block sit in K
+// adjacent lanes and the exclusive product is formed with K-1 shuffles, left to right.
+// SCAN = false: only lse / conf / row_ce are written; block_scan_kernel finishes the job.
+template <bool SCAN>
+__global__ void __launch_bounds__(ROW_THREADS) row_kernel(const RowParams p) {
+    const int r = blockIdx.x * ROW_THREADS + threadIdx.x;
+    const bool in_range = r < p.T;
+    bool ok = false, bad = false;
+    float c = 1.f, ce = 0.f;
+    if (in_range) {
+        // merge the per-split (max, sum-exp) pairs in split order
+        float m = -INFINITY;
+        for (int s = 0; s < p.S; ++s) m = fmaxf(m, p.part_m[static_cast<size_t>(s) * p.T + r]);
+        float l = 0.f;
+        for (int s = 0; s < p.S; ++s)
+            l += p.part_l[static_cast<size_t>(s) * p.T + r] * expf(p.part_m[static_cast<size_t>(s) * p.T + r] - m);
+        const float lse = m + logf(l);
+        p.lse[r] = lse;
+        const long long y = p.labels[r];
+        const bool mask = (p.valid == nullptr) || (p.valid[r] != 0);
+        const bool y_ok = (y >= 0 && y < p.V);
+        ok = mask && y_ok;
+        bad = mask && !y_ok;
+        if (ok) {
+            const float zy = p.z_label[r];
+            ce = lse - zy;
+            c = p.conf_ext ? p.conf_ext[r] : expf(zy - lse);   // Eq. 9
+        }
+        p.conf[r] = c;
+    }
+    if (SCAN) {
+        // Eq. 10: weight_k = ((1 * c_0) * c_1) ... * c_{k-1}; invalid rows carry the factor 1
+        const int lane = threadIdx.x & 31;
+        const int k = lane & (p.K - 1);
+        const int base = lane - k;
+        float run = 1.f;
+        for (int j = 0; j + 1 < p.K; ++j) {
+            const float cj = __shfl_sync(0xffffffffu, c, base + j);
+            if (k > j) run = run * cj;
+        }
+        const float w = ok ? run : 0.f;
+        if (in_range) p.weight[r] = w;
+        block_reduce_store(static_cast<double>(w) * static_cast<double>(ce), w, static_cast<double>(w) * c,
+                           ok ? 1 : 0, bad ? 1 : 0, &p.partials[blockIdx.x]);
+    } else {
+        if (in_range) p.row_ce[r] = ce;
+    }
+}
+
+// General K (not a power of two, or > 32): one thread per draft block, sequential product.
+__global__ void __launch_bounds__(ROW_THREADS) block_scan_kernel(const RowParams p) {
+    const int b = blockIdx.x * ROW_THREADS + threadIdx.x;
+    const int B = p.T / p.K;
+    double loss = 0.0, sw = 0.0, swc = 0.0;
+    long long nv = 0, nb = 0;
+    if (b < B) {
+        float run = 1.f;
+        for (int k = 0; k < p.K; ++k) {
+            const int r = b * p.K + k;
+            const long long y = p.labels[r];
+            const bool mask = (p.valid == nullptr) || (p.valid[r] != 0);
+            const bool y_ok = (y >= 0 && y < p.V);
+            const bool ok = mask && y_ok;
+            const float c = p.conf[r];
+            const float w = ok ? run : 0.f;
+            p.weight[r] = w;
+            if (ok) run = run * c;
+            loss += static_cast<double>(w) * static_cast<double>(p.row_ce[r]);
+            sw += w;
+            swc += static_cast<double>(w) * c;
+            nv += ok ? 1 : 0;
+            nb += (mask && !y_ok) ? 1 : 0;
+        }
+    }
+    block_reduce_store(loss, sw, swc, nv, nb, &p.partials[blockIdx.x]);
+}
+
+struct StatsOut {   // mirrors cat_stats
+    long long n_valid, n_bad_labels;
+    float sum_weight, est_accept_len;
+    int device_status, reserved;
+};
+
+// Single CTA: adds the per-CTA partials in index order and writes loss = sum / N (Eq. 11).
+__global__ void __launch_bounds__(ROW_THREADS) finalize_kernel(const CtaPartial* partials, int n_partials, int n_blocks,
+                                                               float* loss, StatsOut* stats, const int* status) {
+    __shared__ CtaPartial sh[ROW_THREADS];
+    CtaPartial acc = {0.0, 0.0, 0.0, 0, 0};
+    for (int i = threadIdx.x; i < n_partials; i += ROW_THREADS) {
+        const CtaPartial q = partials[i];
+        acc.loss += q.loss; acc.sum_w += q.sum_w; acc.sum_wc += q.sum_wc; acc.n_valid += q.n_valid; acc.n_bad += q.n_bad;
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int off = ROW_THREADS / 2; off > 0; off >>= 1) {
+        if (threadIdx.x < off) {
+            CtaPartial a = sh[threadIdx.x];
+            const CtaPartial b = sh[threadIdx.x + off];
+            a.loss += b.loss; a.sum_w += b.sum_w; a.sum_wc += b.sum_wc; a.n_valid += b.n_valid; a.n_bad += b.n_bad;
+            sh[threadIdx.x] = a;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const CtaPartial t = sh[0];
+        *loss = t.n_valid > 0 ? static_cast<float>(t.loss / static_cast<double>(t.n_valid)) : 0.f;
+        if (stats) {
+            stats->n_valid = t.n_valid;
+            stats->n_bad_labels = t.n_bad;
+            stats->sum_weight = static_cast<float>(t.sum_w);
+            stats->est_accept_len = n_blocks > 0 ? static_cast<float>(t.sum_wc / n_blocks) : 0.f;
+            stats->device_status = *status;
+            stats->reserved = 0;
+        }
+    }
+}
+
+// Backward set-up, single CTA: N = number of valid rows, scale = g / N (0 when N = 0).
+__global__ void __launch_bounds__(1024) bwd_scale_kernel(const long long* labels, const unsigned char* valid, int T, int V,
+                                                         const float* grad_loss, float* scale) {
+    __shared__ int sh[32];
+    int n = 0;
+    for (int r = threadIdx.x; r < T; r += 1024) {
+        const long long y = labels[r];
+        n += ((valid == nullptr || valid[r] != 0) && y >= 0 && y < V) ? 1 : 0;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) n += __shfl_down_sync(0xffffffffu, n, off);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int tot = 0;
+        for (int w = 0; w < 32; ++w) tot += sh[w];
+        const float g = grad_loss ? *grad_loss : 1.f;
+        *scale = tot > 0 ? g / static_cast<float>(tot) : 0.f;
+    }
+}
+
+}  // namespace rows
+}  // namespace cat

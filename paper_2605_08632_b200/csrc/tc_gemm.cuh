@@ -1,0 +1,494 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a: TMA-fed shared-memory ring,
+// tcgen05.mma with fp32 accumulators in tensor memory (two 128x256 accumulators, so the
+// epilogue of one tile overlaps the main loop of the next), and pluggable epilogues that
+// read the accumulators straight from TMEM, one output row per thread.
+//
+// The three dense contractions of the CAT loss all run through this kernel:
+//   logits        z  = H W^T          A = H  (K-major),  B = W   (K-major)   forward + recompute
+//   dW slice      dW = dz^T H         A = dz (MN-major), B = H   (MN-major)
+//   dH            dH += dz W          A = dz (K-major),  B = W   (MN-major)
+// Operands are never transposed in memory: MN-major operands are described to the tensor
+// core through the shared-memory descriptor's leading/stride offsets and the instruction
+// descriptor's major bits.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA
+// issuer (one lane), warps 2-5 = epilogue (TMEM lane quarter = warp index mod 4).
+// Every mbarrier wait is bounded; when one expires the CTA raises an abort flag, records
+// CAT_ERR_TIMEOUT in the status word, drains what it issued, frees its TMEM and returns.
+#pragma once
+#include "ptx.cuh"
+#include <cuda_bf16.h>
+
+namespace cat {
+namespace tc {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int MN_ATOM_BYTES = 64 * BK * 2;                // one 64(MN) x BK box of an MN-major operand
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr int STATUS_TIMEOUT = -8;                        // CAT_ERR_TIMEOUT
+constexpr float LOG2E = 1.4426950408889634f;
+
+// Static tile schedule shared by the three roles of a CTA.
+struct Sched {
+    int num_m_tiles;   // tiles of BM rows of the output
+    int num_n_tiles;   // tiles of BN columns of the output
+    int num_kb;        // blocks of BK along the contraction
+    int n_groups;      // column groups per m-tile: one item = (m-tile, group); a group is a run of n-tiles
+    int band_m;        // m-tiles per band when m runs fastest (keeps a band of A rows L2-resident)
+    int n_fastest;     // 1: items ordered group-fastest within an m-tile; 0: m-fastest within (band, group)
+    int n_items;       // num_m_tiles * n_groups
+};
+
+__device__ __forceinline__ void decode_item(const Sched& s, int item, int& m_tile, int& group, int& n_begin, int& n_end) {
+    if (s.n_fastest) {
+        m_tile = item / s.n_groups;
+        group = item - m_tile * s.n_groups;
+    } else {
+        const int per_band = s.band_m * s.n_groups;
+        const int band = item / per_band;
+        const int rem = item - band * per_band;
+        const int mb = min(s.band_m, s.num_m_tiles - band * s.band_m);
+        group = rem / mb;
+        m_tile = band * s.band_m + (rem - group * mb);
+    }
+    n_begin = static_cast<int>((static_cast<long long>(group) * s.num_n_tiles) / s.n_groups);
+    n_end = static_cast<int>((static_cast<long long>(group + 1) * s.num_n_tiles) / s.n_groups);
+}
+
+struct Ctl {
+    unsigned long long full[STAGES];
+    unsigned long long empty[STAGES];
+    unsigned long long tfull[2];
+    unsigned long long tempty[2];
+    unsigned long long drain;
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort, int* status,
+                                             unsigned long long limit_ns = WAIT_LIMIT_NS) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    uint32_t spins = 0;
+    while (true) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*abort) return false;
+            const unsigned long long now = ptx::globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > limit_ns) {
+                *abort = 1;
+                atomicExch(status, STATUS_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Epilogues.  Each epilogue thread owns output row (m_tile*BM + row_in_tile) and walks the
+// 256 accumulator columns of a tile in chunks of 32 (one tcgen05.ld each).  taddr is the TMEM
+// address of column 0 of the tile for this warp's lane quarter.
+// ------------------------------------------------------------------------------------------
+
+// Forward: online max / sum-exp over the vocabulary (softmax partition function of Eq. 11's
+// log P), and the label logit z[r, y_r] picked from the accumulator chunk that holds it.
+struct EpiFwd {
+    struct Params {
+        const long long* labels;   // [T]
+        float* part_m;             // [n_groups][T] running max of each (row, vocabulary split)
+        float* part_l;             // [n_groups][T] sum exp(z - max)
+        float* z_label;            // [T]
+        int T;
+        int V;
+    };
+    struct State {
+        float m_run, l_run;
+        int y;
+        int row;
+    };
+    __device__ static __forceinline__ void begin_item(const Params& p, State& s, int m_tile, int row_in_tile) {
+        s.row = m_tile * BM + row_in_tile;
+        s.m_run = -INFINITY;
+        s.l_run = 0.f;
+        s.y = -1;
+        if (s.row < p.T) {
+            const long long y = p.labels[s.row];
+            if (y >= 0 && y < p.V) s.y = static_cast<int>(y);
+        }
+    }
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
+        const int col0 = n_tile * BN;
+        const int ncols = min(BN, p.V - col0);
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            if (c * 32 >= ncols) break;
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + c * 32, v);
+            ptx::tmem_ld_wait();
+            float f[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+            const int live = ncols - c * 32;
+            if (live < 32) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i >= live) f[i] = -INFINITY;
+            }
+            const int rel = s.y - (col0 + c * 32);
+            if (rel >= 0 && rel < 32) {
+                float zy = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i == rel) zy = f[i];
+                p.z_label[s.row] = zy;
+            }
+            float cmax = f[0];
+#pragma unroll
+            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, f[i]);
+            const float m_new = fmaxf(s.m_run, cmax);
+            const float mb = m_new * LOG2E;
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sum += ptx::ex2_approx(fmaf(f[i], LOG2E, -mb));
+            s.l_run = fmaf(s.l_run, ptx::ex2_approx((s.m_run - m_new) * LOG2E), sum);
+            s.m_run = m_new;
+        }
+    }
+    __device__ static __forceinline__ void end_item(const Params& p, const State& s, int group) {
+        if (s.row < p.T) {
+            p.part_m[static_cast<size_t>(group) * p.T + s.row] = s.m_run;
+            p.part_l[static_cast<size_t>(group) * p.T + s.row] = s.l_run;
+        }
+    }
+};
+
+// Backward recompute: dz[r, v] = weight_r * (exp(z - lse_r) - [v == y_r]) as a bf16 tile of the
+// current vocabulary slab (the scalar g/N is applied later, in fp32, by the dH / dW epilogues).
+struct EpiDz {
+    struct Params {
+        const long long* labels;   // [T]
+        const unsigned char* valid;  // [T] or nullptr
+        const float* lse;          // [T]
+        const float* weight;       // [T]
+        __nv_bfloat16* dz;         // [T][ld] slab, column 0 = vocabulary index v0
+        long long ld;
+        int T;
+        int V;
+        int v0;
+    };
+    struct State {
+        float w, l2;
+        int y_rel;
+        int row;
+    };
+    __device__ static __forceinline__ void begin_item(const Params& p, State& s, int m_tile, int row_in_tile) {
+        s.row = m_tile * BM + row_in_tile;
+        s.w = 0.f;
+        s.l2 = INFINITY;
+        s.y_rel = -1;
+        if (s.row < p.T) {
+            const long long y = p.labels[s.row];
+            const bool ok = (p.valid == nullptr || p.valid[s.row] != 0) && y >= 0 && y < p.V;
+            if (ok) {
+                s.w = p.weight[s.row];
+                s.l2 = p.lse[s.row] * LOG2E;
+                s.y_rel = static_cast<int>(y) - p.v0;
+            }
+        }
+    }
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
+        const int col0 = n_tile * BN;
+        const int ncols = min(BN, p.V - p.v0 - col0);
+        __nv_bfloat16* out = p.dz + static_cast<size_t>(s.row) * p.ld + col0;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + c * 32, v);
+            ptx::tmem_ld_wait();
+            float f[32];
+            const int live = ncols - c * 32;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float pz = ptx::ex2_approx(fmaf(__uint_as_float(v[i]), LOG2E, -s.l2));
+                f[i] = (i < live) ? s.w * pz : 0.f;
+            }
+            const int rel = s.y_rel - (col0 + c * 32);
+            if (rel >= 0 && rel < 32) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i == rel) f[i] -= s.w;
+            }
+            if (s.row < p.T) {
+                uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 pk;
+                    __nv_bfloat162 b0 = __floats2bfloat162_rn(f[q * 8 + 0], f[q * 8 + 1]);
+                    __nv_bfloat162 b1 = __floats2bfloat162_rn(f[q * 8 + 2], f[q * 8 + 3]);
+                    __nv_bfloat162 b2 = __floats2bfloat162_rn(f[q * 8 + 4], f[q * 8 + 5]);
+                    __nv_bfloat162 b3 = __floats2bfloat162_rn(f[q * 8 + 6], f[q * 8 + 7]);
+                    pk.x = *reinterpret_cast<uint32_t*>(&b0);
+                    pk.y = *reinterpret_cast<uint32_t*>(&b1);
+                    pk.z = *reinterpret_cast<uint32_t*>(&b2);
+                    pk.w = *reinterpret_cast<uint32_t*>(&b3);
+                    dst[q] = pk;
+                }
+            }
+        }
+    }
+    __device__ static __forceinline__ void end_item(const Params&, const State&, int) {}
+};
+
+// Plain output: out = add + alpha * acc, fp32 or bf16, with optional fp32/bf16 addend
+// (dH accumulation across vocabulary slabs, accumulate_dW).
+struct EpiOut {
+    struct Params {
+        const float* alpha;            // device scalar or nullptr (= 1)
+        const float* add_f32;          // [M][ld_add] or nullptr
+        const __nv_bfloat16* add_bf16; // [M][ld_add] or nullptr
+        float* out_f32;                // [M][ld_out] or nullptr
+        __nv_bfloat16* out_bf16;       // [M][ld_out] or nullptr
+        long long ld_add, ld_out;
+        int M, N;
+    };
+    struct State {
+        float alpha;
+        int row;
+    };
+    __device__ static __forceinline__ void begin_item(const Params& p, State& s, int m_tile, int row_in_tile) {
+        s.row = m_tile * BM + row_in_tile;
+        s.alpha = p.alpha ? *p.alpha : 1.f;
+    }
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
+        const int col0 = n_tile * BN;
+        const bool row_ok = s.row < p.M;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            if (col0 + c * 32 >= p.N) break;
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + c * 32, v);
+            ptx::tmem_ld_wait();
+            if (!row_ok) continue;
+            const int cbase = col0 + c * 32;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int col = cbase + q * 8;
+                if (col + 8 > p.N) continue;   // N is a multiple of 8: groups are all-in or all-out
+                float f[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] = s.alpha * __uint_as_float(v[q * 8 + i]);
+                if (p.add_f32) {
+                    const float4* a = reinterpret_cast<const float4*>(p.add_f32 + static_cast<size_t>(s.row) * p.ld_add + col);
+                    const float4 a0 = a[0], a1 = a[1];
+                    f[0] += a0.x; f[1] += a0.y; f[2] += a0.z; f[3] += a0.w;
+                    f[4] += a1.x; f[5] += a1.y; f[6] += a1.z; f[7] += a1.w;
+                } else if (p.add_bf16) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(p.add_bf16 + static_cast<size_t>(s.row) * p.ld_add + col);
+                    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+                        f[2 * i] += t.x;
+                        f[2 * i + 1] += t.y;
+                    }
+                }
+                if (p.out_f32) {
+                    float4* o = reinterpret_cast<float4*>(p.out_f32 + static_cast<size_t>(s.row) * p.ld_out + col);
+                    o[0] = make_float4(f[0], f[1], f[2], f[3]);
+                    o[1] = make_float4(f[4], f[5], f[6], f[7]);
+                } else {
+                    uint4 pk;
+                    __nv_bfloat162 b0 = __floats2bfloat162_rn(f[0], f[1]);
+                    __nv_bfloat162 b1 = __floats2bfloat162_rn(f[2], f[3]);
+                    __nv_bfloat162 b2 = __floats2bfloat162_rn(f[4], f[5]);
+                    __nv_bfloat162 b3 = __floats2bfloat162_rn(f[6], f[7]);
+                    pk.x = *reinterpret_cast<uint32_t*>(&b0);
+                    pk.y = *reinterpret_cast<uint32_t*>(&b1);
+                    pk.z = *reinterpret_cast<uint32_t*>(&b2);
+                    pk.w = *reinterpret_cast<uint32_t*>(&b3);
+                    *reinterpret_cast<uint4*>(p.out_bf16 + static_cast<size_t>(s.row) * p.ld_out + col) = pk;
+                }
+            }
+        }
+    }
+    __device__ static __forceinline__ void end_item(const Params&, const State&, int) {}
+};
+
+// ------------------------------------------------------------------------------------------
+// The kernel.  tmA / tmB are 2-D tiled tensor maps with 128-byte swizzle:
+//   K-major operand  [rows = M or N][cols = K]: box {BK, BM or BN}, one box per stage;
+//   MN-major operand [rows = K][cols = M or N]: box {64, BK}, BM/64 or BN/64 boxes per stage.
+// Rows/columns past the tensor's extent are zero-filled by TMA, which makes ragged M, N and K
+// contribute exact zeros.
+// ------------------------------------------------------------------------------------------
+template <int A_MN, int B_MN, class Epi>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const Sched sched, const typename Epi::Params ep, int* status) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ Ctl ctl;
+    const uint32_t ring = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        ptx::prefetch_tmap(&tmA);
+        ptx::prefetch_tmap(&tmB);
+        for (int i = 0; i < STAGES; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctl.full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctl.empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctl.tfull[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctl.tempty[i]), NUM_THREADS - 64);
+        }
+        ptx::mbar_init(ptx::smem_u32(&ctl.drain), 1);
+        ctl.abort = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc<TMEM_COLS>(ptx::smem_u32(&ctl.tmem_base));
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = ctl.tmem_base;
+    volatile int* abort = &ctl.abort;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, issued = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < sched.n_items && ok; item += gridDim.x) {
+                int m_tile, group, n_begin, n_end;
+                decode_item(sched, item, m_tile, group, n_begin, n_end);
+                for (int n = n_begin; n < n_end && ok; ++n) {
+                    for (int kb = 0; kb < sched.num_kb; ++kb) {
+                        if (!wait_bounded(ptx::smem_u32(&ctl.empty[stage]), phase ^ 1u, abort, status)) { ok = false; break; }
+                        const uint32_t full = ptx::smem_u32(&ctl.full[stage]);
+                        ptx::mbar_arrive_expect_tx(full, STAGE_BYTES);
+                        const uint32_t a_dst = ring + stage * STAGE_BYTES;
+                        const uint32_t b_dst = a_dst + A_STAGE_BYTES;
+                        if (A_MN) {
+#pragma unroll
+                            for (int j = 0; j < BM / 64; ++j)
+                                ptx::tma_load_2d(a_dst + j * MN_ATOM_BYTES, &tmA, m_tile * BM + j * 64, kb * BK, full);
+                        } else {
+                            ptx::tma_load_2d(a_dst, &tmA, kb * BK, m_tile * BM, full);
+                        }
+                        if (B_MN) {
+#pragma unroll
+                            for (int j = 0; j < BN / 64; ++j)
+                                ptx::tma_load_2d(b_dst + j * MN_ATOM_BYTES, &tmB, n * BN + j * 64, kb * BK, full);
+                        } else {
+                            ptx::tma_load_2d(b_dst, &tmB, kb * BK, n * BN, full);
+                        }
+                        ++issued;
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                // aborted: let the copies already issued land before the CTA exits
+                const uint32_t back = issued < STAGES ? issued : STAGES;
+                for (uint32_t i = 0; i < back; ++i) {
+                    const uint32_t q = issued - 1 - i;
+                    wait_bounded(ptx::smem_u32(&ctl.full[q % STAGES]), (q / STAGES) & 1u, abort, status, 20000000ull);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN, A_MN, B_MN);
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < sched.n_items && ok; item += gridDim.x) {
+                int m_tile, group, n_begin, n_end;
+                decode_item(sched, item, m_tile, group, n_begin, n_end);
+                for (int n = n_begin; n < n_end && ok; ++n) {
+                    if (!wait_bounded(ptx::smem_u32(&ctl.tempty[acc]), acc_phase ^ 1u, abort, status)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t d_tmem = tmem + acc * BN;
+                    for (int kb = 0; kb < sched.num_kb; ++kb) {
+                        if (!wait_bounded(ptx::smem_u32(&ctl.full[stage]), phase, abort, status)) { ok = false; break; }
+                        ptx::tc_fence_after();
+                        const uint32_t a_base = ring + stage * STAGE_BYTES;
+                        const uint32_t b_base = a_base + A_STAGE_BYTES;
+#pragma unroll
+                        for (int j = 0; j < BK / 16; ++j) {
+                            // K-major: 16 elements = 32 bytes further inside the 128-byte swizzle row.
+                            // MN-major: 16 k-rows = two 8-row swizzle atoms (2048 bytes) further.
+                            const uint64_t adesc = A_MN ? ptx::smem_desc_sw128(a_base + j * 2048, MN_ATOM_BYTES, 1024)
+                                                        : ptx::smem_desc_sw128(a_base + j * 32, 16, 1024);
+                            const uint64_t bdesc = B_MN ? ptx::smem_desc_sw128(b_base + j * 2048, MN_ATOM_BYTES, 1024)
+                                                        : ptx::smem_desc_sw128(b_base + j * 32, 16, 1024);
+                            ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
+                        }
+                        ptx::umma_commit(ptx::smem_u32(&ctl.empty[stage]));   // frees the stage once these MMAs have read it
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    ptx::umma_commit(ptx::smem_u32(&ctl.tfull[acc]));         // accumulator complete
+                    acc ^= 1u;
+                    if (acc == 0) acc_phase ^= 1u;
+                }
+            }
+            if (!ok) {
+                // aborted: make sure no MMA is still in flight before TMEM is freed
+                ptx::umma_commit(ptx::smem_u32(&ctl.drain));
+                wait_bounded(ptx::smem_u32(&ctl.drain), 0, abort, status, 20000000ull);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        typename Epi::State st;
+        for (int item = blockIdx.x; item < sched.n_items && ok; item += gridDim.x) {
+            int m_tile, group, n_begin, n_end;
+            decode_item(sched, item, m_tile, group, n_begin, n_end);
+            Epi::begin_item(ep, st, m_tile, row_in_tile);
+            for (int n = n_begin; n < n_end; ++n) {
+                ok = wait_bounded(ptx::smem_u32(&ctl.tfull[acc]), acc_phase, abort, status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ptx::tc_fence_after();
+                Epi::tile(ep, st, n, lane_base + acc * BN);
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(ptx::smem_u32(&ctl.tempty[acc]));
+                acc ^= 1u;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+            if (ok) Epi::end_item(ep, st, group);
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc<TMEM_COLS>(tmem);
+    }
+}
+
+}  // namespace tc
+}  // namespace cat

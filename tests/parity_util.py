@@ -1,0 +1,93 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C ABI, run the
+oracle on the same seeded batch, and compare element by element with the stated tolerances.
+
+Tolerances (bf16 inputs, fp32 accumulation): loss relative error <= 1e-3, per-tensor gradient
+relative L2 error <= 1e-2.  fp32 config: loss 1e-5, gradients 1e-4, confidences 1e-5.
+The CAT weight vector must equal, bit for bit, the binary32 left-to-right product of the
+GPU's own confidences (the bit-exact claim), and agree with the fp64 oracle's weights within
+rounding; products that underflow binary32 (~V^-k for k large) are compared with an absolute
+floor.
+"""
+import numpy as np
+import torch
+
+from oracle import cat_oracle as O
+from paper_2605_08632_b200.api import CatLoss
+
+TOL = {
+    torch.bfloat16: dict(loss=1e-3, grad=1e-2, lse=2e-3, conf=5e-3),
+    torch.float32: dict(loss=1e-5, grad=1e-4, lse=1e-5, conf=1e-5),
+}
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
+    den = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / den) if den > 0 else float(np.linalg.norm(a))
+
+
+def run_gpu(batch, slab_mib=0, g=None, conf_ext=None, dW_dtype=torch.float32, use_valid=True, accumulate_into=None):
+    dev = torch.device("cuda")
+    H, W = batch.H.to(dev), batch.W.to(dev)
+    labels = batch.labels.to(dev)
+    valid = batch.valid.to(dev) if use_valid else None
+    cl = CatLoss(batch.T, batch.d, batch.V, batch.K, dtype=batch.torch_dtype, dW_dtype=dW_dtype, slab_mib=slab_mib)
+    ce = None if conf_ext is None else torch.as_tensor(conf_ext, dtype=torch.float32, device=dev)
+    gl = None if g is None else torch.tensor([g], dtype=torch.float32, device=dev)
+    cl.forward(H, W, labels, valid, ce)
+    acc = False
+    if accumulate_into is not None:
+        cl.dW.copy_(torch.as_tensor(accumulate_into, device=dev).to(dW_dtype))
+        acc = True
+    cl.backward(H, W, labels, valid, gl, accumulate_dW=acc)
+    torch.cuda.synchronize()
+    st = cl.fwd_stats()
+    out = dict(loss=float(cl.loss.item()), lse=cl.lse.cpu().numpy(), conf=cl.conf.cpu().numpy(),
+               weight=cl.weight.cpu().numpy(), dH=cl.dH.float().cpu().numpy(), dW=cl.dW.float().cpu().numpy(),
+               stats=st, bwd_status=cl.bwd_status(), obj=cl)
+    return out
+
+
+def run_oracle(batch, g=1.0, conf_ext=None, use_valid=True):
+    fwd, dH, dW = O.cat_forward_backward(batch.H, batch.W, batch.labels, batch.valid if use_valid else None, batch.K,
+                                         conf_ext=conf_ext, g=g)
+    return fwd, dH, dW
+
+
+def check_forward(gpu, fwd, K, dtype, V):
+    tol = TOL[dtype]
+    ok = fwd["eff_valid"]
+    assert gpu["stats"].device_status == 0
+    assert gpu["stats"].n_valid == fwd["n_valid"]
+    assert abs(gpu["loss"] - fwd["loss"]) <= tol["loss"] * abs(fwd["loss"]) + 1e-12, (gpu["loss"], fwd["loss"])
+    assert np.max(np.abs(gpu["lse"] - fwd["lse"]) / np.maximum(1.0, np.abs(fwd["lse"]))) <= tol["lse"]
+    # confidences: relative, with an absolute floor far below anything that matters
+    cerr = np.abs(gpu["conf"] - fwd["conf"]) / np.maximum(np.abs(fwd["conf"]), 1e-30)
+    assert np.max(cerr) <= tol["conf"], np.max(cerr)
+    assert np.all(gpu["conf"][~ok] == 1.0)
+    # bit-exact: weights are the binary32 left-to-right product of the GPU's own confidences
+    w32 = O.cat_weights_f32(gpu["conf"].astype(np.float32), ok, K)
+    assert gpu["weight"].tobytes() == w32.tobytes()
+    # and they agree with the fp64 oracle's weights (K-1 factors, each within tol["conf"])
+    werr = np.abs(gpu["weight"].astype(np.float64) - fwd["weight"])
+    assert np.all(werr <= K * tol["conf"] * fwd["weight"] + 1e-37), np.max(werr / np.maximum(fwd["weight"], 1e-37))
+    assert np.all(gpu["weight"][~ok] == 0.0)
+
+
+def check_backward(gpu, fwd, dH, dW, K, dtype, per_position=True):
+    tol = TOL[dtype]
+    assert gpu["bwd_status"] == 0
+    assert rel_l2(gpu["dH"], dH) <= tol["grad"], rel_l2(gpu["dH"], dH)
+    assert rel_l2(gpu["dW"], dW) <= tol["grad"], rel_l2(gpu["dW"], dW)
+    ok = fwd["eff_valid"]
+    assert not gpu["dH"][~ok].any()
+    if per_position:
+        # the loss is dominated by position 0; compare dH separately for every position in the block
+        T = dH.shape[0]
+        gH, oH = gpu["dH"].reshape(T // K, K, -1), dH.reshape(T // K, K, -1)
+        top = np.linalg.norm(oH[:, 0])
+        for k in range(K):
+            nk = np.linalg.norm(oH[:, k])
+            if nk > 1e-30 and nk > 1e-25 * top:
+                e = np.linalg.norm(gH[:, k] - oH[:, k]) / nk
+                assert e <= 2 * tol["grad"], (k, e)

@@ -1,0 +1,138 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs.  Reduced-T versions of the five configs keep d, V and K at full size and
+span several 128-row tiles with a ragged tail; edge cases cover the degenerate shapes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cat_oracle as O
+from paper_2605_08632_b200 import synth
+from paper_2605_08632_b200 import binding as B
+from paper_2605_08632_b200.api import CatLoss
+
+from parity_util import TOL, check_backward, check_forward, rel_l2, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_check(batch, **kw):
+    gpu = run_gpu(batch, **{k: v for k, v in kw.items() if k in ("slab_mib", "g", "conf_ext", "use_valid")})
+    fwd, dH, dW = run_oracle(batch, g=kw.get("g") or 1.0, conf_ext=kw.get("conf_ext"), use_valid=kw.get("use_valid", True))
+    check_forward(gpu, fwd, batch.K, batch.torch_dtype, batch.V)
+    check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype)
+    return gpu, fwd
+
+
+def test_config1_fp32_full_size_bit_exact_weights_and_determinism():
+    batch = synth.make_batch(1)
+    gpu, fwd = _full_check(batch)
+    again = run_gpu(batch)
+    for key in ("lse", "conf", "weight", "dH", "dW"):
+        assert gpu[key].tobytes() == again[key].tobytes(), key
+    assert gpu["loss"] == again["loss"]
+
+
+@pytest.mark.parametrize("cfg,T", [(2, 600), (3, 400), (4, 520), (41, 520), (5, 448)])
+def test_reduced_configs_full_d_V_K(cfg, T):
+    batch = synth.make_batch(cfg, T=T - T % synth.CONFIGS[cfg].K)
+    gpu, fwd = _full_check(batch)
+    if cfg == 41:
+        assert fwd["weight"].reshape(-1, batch.K)[:, 1:].max() > 0.1     # later positions carry real weight
+
+
+def test_bf16_run_twice_is_bitwise_identical():
+    batch = synth.make_batch(2, T=512, V=20000)
+    a, b = run_gpu(batch), run_gpu(batch)
+    for key in ("lse", "conf", "weight", "dH", "dW"):
+        assert a[key].tobytes() == b[key].tobytes(), key
+
+
+@pytest.mark.parametrize("dtype_cfg", [2, 1])
+def test_many_vocabulary_slabs_and_ragged_everything(dtype_cfg):
+    # V not a multiple of the tile, T not a multiple of the tile, d one partial k-block beyond a multiple of 64
+    batch = synth.make_batch(41 if dtype_cfg == 2 else 1, T=392, d=200, V=5000, K=8)
+    if dtype_cfg == 1:
+        batch.valid[5] = 0; batch.valid[100:108] = 0
+    gpu, fwd = _full_check(batch, slab_mib=1)
+    assert B.cat_loss_workspace_bytes(gpu["obj"].shape, 1) < 3 << 20
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 16, 32, 40])
+def test_block_lengths(K):
+    batch = synth.make_batch(41, T=K * 24, d=128, V=1024, K=K)
+    _full_check(batch)
+
+
+def test_tiny_shapes():
+    for (T, d, V, K) in [(8, 8, 40, 8), (4, 72, 300, 4), (130, 64, 256, 2)]:
+        batch = synth.make_batch(41, T=T, d=d, V=V, K=K)
+        _full_check(batch)
+
+
+def test_all_rows_invalid_gives_zero_loss_and_gradients():
+    batch = synth.make_batch(2, T=256, d=128, V=1000)
+    batch.valid[:] = 0
+    gpu = run_gpu(batch)
+    assert gpu["loss"] == 0.0 and gpu["stats"].n_valid == 0
+    assert not gpu["dH"].any() and not gpu["dW"].any() and not gpu["weight"].any()
+
+
+def test_out_of_range_labels_are_counted_and_ignored():
+    batch = synth.make_batch(2, T=256, d=128, V=1000)
+    batch.labels[3] = 1000; batch.labels[17] = -5; batch.labels[200] = 2 ** 40
+    gpu, fwd = _full_check(batch)
+    assert gpu["stats"].n_bad_labels == 3 and gpu["stats"].n_valid == 253
+
+
+def test_upstream_scalar_external_confidence_and_no_mask_pointer():
+    batch = synth.make_batch(4, T=512, d=256, V=3000)
+    rng = np.random.default_rng(5)
+    conf_ext = rng.random(512).astype(np.float32)
+    gpu, fwd = _full_check(batch, g=0.1, conf_ext=conf_ext)            # beta of Eq. 12 as the upstream scalar
+    batch2 = synth.make_batch(2, T=512, d=256, V=3000)
+    _full_check(batch2, use_valid=False)
+    # Eq. 8 estimate reported in the stats
+    est = float((fwd["weight"] * fwd["conf"] * fwd["eff_valid"]).reshape(-1, batch.K).sum(1).mean())
+    assert abs(gpu["stats"].est_accept_len - est) <= 1e-3 * est
+
+
+def test_bf16_dW_output_and_accumulate():
+    batch = synth.make_batch(41, T=384, d=256, V=2048)
+    fwd, dH, dW = run_oracle(batch)
+    gpu = run_gpu(batch, dW_dtype=torch.bfloat16)
+    assert rel_l2(gpu["dW"], dW) <= 1.5e-2
+    base = np.random.default_rng(6).standard_normal(dW.shape).astype(np.float32) * float(np.abs(dW).max())
+    gpu = run_gpu(batch, accumulate_into=base)
+    assert rel_l2(gpu["dW"] - base, dW) <= 2e-2
+    assert rel_l2(gpu["dW"], dW + base) <= 1e-4
+
+
+def test_row_pitch_larger_than_d():
+    batch = synth.make_batch(41, T=256, d=192, V=1536)
+    dev = torch.device("cuda")
+    ld = 256
+    Hp = torch.zeros(batch.T, ld, dtype=torch.bfloat16, device=dev); Hp[:, :192] = batch.H.to(dev)
+    Wp = torch.zeros(batch.V, ld, dtype=torch.bfloat16, device=dev); Wp[:, :192] = batch.W.to(dev)
+    Hp[:, 192:] = 7.0; Wp[:, 192:] = 7.0         # padding must never be read as data
+    cl = CatLoss(batch.T, 192, batch.V, batch.K)
+    cl.shape.ldH = ld; cl.shape.ldW = ld
+    cl.dH = torch.full((batch.T, ld), 3.0, dtype=torch.bfloat16, device=dev)
+    cl.dW = torch.full((batch.V, ld), 3.0, dtype=torch.float32, device=dev)
+    labels, valid = batch.labels.to(dev), batch.valid.to(dev)
+    cl.forward(Hp, Wp, labels, valid)
+    cl.backward(Hp, Wp, labels, valid)
+    torch.cuda.synchronize()
+    fwd, dH, dW = run_oracle(batch)
+    assert abs(cl.loss.item() - fwd["loss"]) <= 1e-3 * fwd["loss"]
+    assert rel_l2(cl.dH[:, :192].float().cpu().numpy(), dH) <= 1e-2
+    assert rel_l2(cl.dW[:, :192].cpu().numpy(), dW) <= 1e-2
+    assert torch.all(cl.dH[:, 192:] == 3.0) and torch.all(cl.dW[:, 192:] == 3.0)
+
+
+def test_errors_on_gpu_box_leave_context_usable():
+    s = B.make_shape(64, 128, 512, 8, B.CAT_BF16)
+    x = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.CatError) as e:
+        B.cat_loss_fwd(s, x, x, x, None, None, x, x, x, x, None, x[:16])
+    assert e.value.code == -5
+    torch.cuda.synchronize()
