@@ -82,12 +82,18 @@ def check_backward(gpu, fwd, dH, dW, K, dtype, per_position=True):
     ok = fwd["eff_valid"]
     assert not gpu["dH"][~ok].any()
     if per_position:
-        # the loss is dominated by position 0; compare dH separately for every position in the block
+        # the loss is dominated by position 0; compare dH separately for every position in the block.
+        # Rows whose label probability is within 1e-3 of 1 are left out of this finer check: their
+        # gradient is w * (sum_{v != y} p_v W_v - (1 - p_y) W_y), and 1 - p_y formed from a binary32
+        # lse carries ~1e-6 absolute rounding, i.e. percent-level relative error on a row whose
+        # gradient is ~1e-5 of a typical one.  They still count in the per-tensor check above.
         T = dH.shape[0]
+        sure = np.exp(np.minimum(fwd["z_label"] - fwd["lse"], 0.0)) > 0.999
+        keep = (~sure).reshape(T // K, K)
         gH, oH = gpu["dH"].reshape(T // K, K, -1), dH.reshape(T // K, K, -1)
         top = np.linalg.norm(oH[:, 0])
         for k in range(K):
-            nk = np.linalg.norm(oH[:, k])
+            nk = np.linalg.norm(oH[keep[:, k], k])
             if nk > 1e-30 and nk > 1e-25 * top:
-                e = np.linalg.norm(gH[:, k] - oH[:, k]) / nk
+                e = np.linalg.norm(gH[keep[:, k], k] - oH[keep[:, k], k]) / nk
                 assert e <= 2 * tol["grad"], (k, e)
