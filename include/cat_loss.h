@@ -56,7 +56,8 @@ typedef enum {
     CAT_ERR_WORKSPACE = -5,  /* workspace NULL or smaller than cat_loss_workspace_bytes()    */
     CAT_ERR_ARCH = -6,       /* current device is not compute capability 10.x                */
     CAT_ERR_CUDA = -7,       /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
-    CAT_ERR_TIMEOUT = -8     /* reported in device_status: a bounded wait in a kernel expired */
+    CAT_ERR_TIMEOUT = -8,    /* reported in device_status: a bounded wait in a kernel expired */
+    CAT_ERR_LIMIT = -9       /* problem needs more scratch than a fixed-capacity entry point owns */
 } cat_status;
 
 typedef enum { CAT_BF16 = 0, CAT_F32 = 1 } cat_dtype;
@@ -138,6 +139,37 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W,
                  const float* lse, const float* weight, const float* grad_loss,
                  void* dH, void* dW, int accumulate_dW,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * cat_loss_fwd for callers that cannot hand over a workspace.  (The paper has no counterpart:
+ * this is a packaging variant of the forward pass above, same arithmetic, same outputs.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated at call time -- a
+ * plug-in living inside another framework's memory pool that has already claimed the whole
+ * GPU, a service whose policy forbids cudaMalloc after start-up because it synchronises the
+ * device and can fail late, or a host with a fixed memory budget.  Such callers own their
+ * inputs and outputs but have nowhere to get scratch from.
+ *
+ * Instead of a caller-supplied workspace, the forward pass's scratch (softmax partials per
+ * row and vocabulary split, label logits, per-CTA loss partials) lives in one array that is
+ * part of the library image: CAT_STATIC_SCRATCH_BYTES of device memory on every GPU that
+ * loads the library, held until the process exits.  The call allocates and frees nothing.
+ *
+ *   - Arguments are those of cat_loss_fwd without `workspace` / `workspace_bytes`.
+ *   - Shapes whose cat_loss_workspace_bytes(shape, 0) exceeds CAT_STATIC_SCRATCH_BYTES are
+ *     refused with CAT_ERR_LIMIT before anything is launched (config 2, T=16384 x V=128256,
+ *     needs 16.7 MB and fits; T=32768 with 128 vocabulary splits does not).
+ *   - The first call on each device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps whatever the last call left in it; the
+ *     words that must start at zero are cleared by every call.  Two calls whose GPU work
+ *     overlaps (different streams, or different host threads) race on it: serialise them.
+ */
+#define CAT_STATIC_SCRATCH_BYTES (32u << 20)
+int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W,
+                        const int64_t* labels, const uint8_t* valid, const float* conf_ext,
+                        float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                        void* cuda_stream);
 
 /*
  * Number of kernels of this library that the given pass (0 = cat_loss_fwd, 1 = cat_loss_bwd)

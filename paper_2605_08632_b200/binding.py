@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.cat_loss_launch_count.argtypes = [ctypes.POINTER(cat_shape), ctypes.c_int]
         L.cat_loss_fwd.restype = ctypes.c_int
         L.cat_loss_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 10 + [vp, sz, vp]
+        L.cat_loss_fwd_static.restype = ctypes.c_int
+        L.cat_loss_fwd_static.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 10 + [vp]
         L.cat_loss_bwd.restype = ctypes.c_int
         L.cat_loss_bwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 9 + [ctypes.c_int, vp, sz, vp]
         _lib = L
@@ -90,6 +92,19 @@ def cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, 
                             _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_loss_fwd")
+
+
+CAT_STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def cat_loss_fwd_static(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats) -> None:
+    """Forward pass that takes no workspace: its scratch is an array built into the library
+    (CAT_STATIC_SCRATCH_BYTES per GPU).  For callers that are not allowed to allocate device
+    memory.  Calls share that array, so do not let two of them overlap on the GPU."""
+    rc = lib().cat_loss_fwd_static(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(conf_ext),
+                                   _ptr(loss), _ptr(lse), _ptr(conf), _ptr(weight), _ptr(stats), _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_loss_fwd_static")
 
 
 def cat_loss_bwd(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace) -> None:

@@ -8,6 +8,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "rowops.cuh"
 #include "simt.cuh"
 #include "tc_gemm.cuh"
@@ -206,6 +208,7 @@ const char* cat_status_string(int status) {
         case CAT_ERR_ARCH: return "current device is not compute capability 10.x";
         case CAT_ERR_CUDA: return "a CUDA call failed";
         case CAT_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case CAT_ERR_LIMIT: return "problem needs more scratch than the built-in static array holds";
         default: return "unknown status";
     }
 }
@@ -418,6 +421,57 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
         }
     }
     return CAT_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Forward pass with built-in scratch, for callers that may not allocate device memory.
+// The array below is part of the module image: each GPU that loads the library carries it
+// until the process ends.  Host code must not use the symbol's name as a pointer (on the host
+// it is only a stand-in); the device address is fetched once per device with
+// cudaGetSymbolAddress and that address is what the kernels receive.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[CAT_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// Set-up, once per device, with that device current: resolve the array's device address.
+int static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_ARCH; }
+    if (dev < 0 || dev >= kMaxDevices) return CAT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return CAT_ERR_CUDA; }
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return CAT_OK;
+}
+}  // namespace
+
+int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                        const float* conf_ext, float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                        void* cuda_stream) {
+    if (!shape) return CAT_ERR_NULL;
+    const int sc = check_shape(shape);
+    if (sc != CAT_OK) return sc;
+    const size_t need = plan_fwd(shape).total;
+    if (need > static_cast<size_t>(CAT_STATIC_SCRATCH_BYTES)) return CAT_ERR_LIMIT;
+    if (!H || !W || !labels || !loss || !lse || !conf || !weight) return CAT_ERR_NULL;
+    int sms = 0;
+    const int dc = check_device(&sms);
+    if (dc != CAT_OK) return dc;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != CAT_OK) return rc;
+    // every call clears the status header it relies on (inside cat_loss_fwd); everything else
+    // in the scratch is fully rewritten before it is read
+    return cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, scratch,
+                        static_cast<size_t>(CAT_STATIC_SCRATCH_BYTES), cuda_stream);
 }
 
 }  // extern "C"
