@@ -71,8 +71,9 @@ typedef struct {
     int32_t in_dtype;  /* cat_dtype of H, W and dH.  CAT_BF16: tensor-core path with
                           fp32 accumulation.  CAT_F32: fp32 FFMA path, fp32 throughout */
     int32_t dW_dtype;  /* cat_dtype of dW: CAT_F32 (default) or CAT_BF16 (bf16 inputs only) */
-    int32_t slab_mib;  /* cap, in MiB, on the backward pass's dz scratch slab; 0 = default
-                          (2048).  Smaller caps mean more, narrower vocabulary slabs.     */
+    int32_t slab_mib;  /* cap, in MiB, on the large scratch slab (dz slab of cat_loss_bwd,
+                          logits slab of cat_loss_fwd_bwd); 0 = default (2048 / 2560).
+                          Smaller caps mean more, smaller slabs.                          */
     int64_t ldH;       /* row pitch of H and dH in elements, >= d                     */
     int64_t ldW;       /* row pitch of W and dW in elements, >= d                     */
 } cat_shape;
@@ -89,7 +90,7 @@ typedef struct {
 
 /*
  * Bytes of scratch the given pass needs for this shape: pass 0 = cat_loss_fwd,
- * pass 1 = cat_loss_bwd.  Returns 0 if the shape is invalid.  The scratch holds the
+ * pass 1 = cat_loss_bwd, pass 2 = cat_loss_fwd_bwd.  Returns 0 if the shape is invalid.  The scratch holds the
  * per-(row, vocabulary split) softmax partials in the forward pass, and in the backward
  * pass one bounded slab of dz (bf16: rows x a slice of the vocabulary, at most about
  * 2 GiB) plus an fp32 dH accumulator when the vocabulary is processed in more than one
@@ -141,6 +142,29 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Forward and backward in one call, without recomputing the logits (same results as
+ * cat_loss_fwd followed by cat_loss_bwd, within rounding).  Rows are processed in slabs of
+ * whole draft blocks.  For each slab the logits GEMM also writes the slab's logits as fp16
+ * (saturating at +-65504); once lse and the CAT weights of the slab's blocks are known
+ * (Eq. 9, Eq. 10) the slab is turned in place into bf16
+ * dz = weight * (exp(z - lse) - one-hot), the label entry taken from the fp32 label logit, and
+ * feeds dH (written once per slab) and dW (accumulated over slabs in fp32).  Executed work is
+ * the 6*T*d*V flops of the three contractions instead of 8*T*d*V; the price is one slab of
+ * logits in the workspace (at most about slab_mib MiB, default 2560, and always at least two
+ * slabs once T exceeds one slab unit, so the T x V logits never exist at once) and fp16 rounding of the stored logits
+ * (relative 2^-11, i.e. about 1e-3 absolute on the logits of the synthetic configs).
+ * Arguments as in cat_loss_fwd and cat_loss_bwd; workspace of
+ * cat_loss_workspace_bytes(shape, 2) bytes; cat_loss_launch_count(shape, 2) kernels.
+ * For CAT_F32 inputs this runs the fp32 forward and backward passes back to back.
+ */
+int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W,
+                     const int64_t* labels, const uint8_t* valid, const float* conf_ext,
+                     const float* grad_loss,
+                     float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                     void* dH, void* dW, int accumulate_dW,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * cat_loss_fwd for callers that cannot hand over a workspace.  (The paper has no counterpart:
  * this is a packaging variant of the forward pass above, same arithmetic, same outputs.)
  *
@@ -172,8 +196,8 @@ int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W,
                         void* cuda_stream);
 
 /*
- * Number of kernels of this library that the given pass (0 = cat_loss_fwd, 1 = cat_loss_bwd)
- * launches for this shape: the logits GEMM, the per-row kernels and the final reduction in
+ * Number of kernels of this library that the given pass (0 = cat_loss_fwd, 1 = cat_loss_bwd,
+ * 2 = cat_loss_fwd_bwd) launches for this shape: the logits GEMM, the per-row kernels and the final reduction in
  * the forward pass; one set-up kernel plus three GEMMs per vocabulary slab in the backward
  * pass.  Host-only; returns 0 for an invalid shape.
  */

@@ -27,6 +27,7 @@ class CatLoss:
             raise ValueError("invalid shape for cat_loss")
         self.ws_fwd = torch.empty(nf, dtype=torch.uint8, device=dev)
         self.ws_bwd = torch.empty(nb, dtype=torch.uint8, device=dev)
+        self._ws_fused = None
         self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
         self.lse = torch.empty(T, dtype=torch.float32, device=dev)
         self.conf = torch.empty(T, dtype=torch.float32, device=dev)
@@ -44,6 +45,18 @@ class CatLoss:
         B.cat_loss_bwd(self.shape, H, W, labels, valid, self.lse, self.weight, grad_loss, self.dH, self.dW,
                        accumulate_dW, self.ws_bwd)
         return self.dH, self.dW
+
+    def forward_backward(self, H, W, labels, valid=None, conf_ext=None, grad_loss=None, accumulate_dW=False):
+        """cat_loss_fwd_bwd: one call, logits kept per row slab instead of recomputed."""
+        if self._ws_fused is None:
+            n = B.cat_loss_workspace_bytes(self.shape, 2)
+            self._ws_fused = torch.empty(n, dtype=torch.uint8, device=self.loss.device)
+        B.cat_loss_fwd_bwd(self.shape, H, W, labels, valid, conf_ext, grad_loss, self.loss, self.lse, self.conf,
+                           self.weight, self.stats, self.dH, self.dW, accumulate_dW, self._ws_fused)
+        return self.loss, self.dH, self.dW
+
+    def fused_status(self) -> int:
+        return int(self._ws_fused[:4].view(torch.int32).item())
 
     def bwd_status(self) -> int:
         return int(self.ws_bwd[:4].view(torch.int32).item())

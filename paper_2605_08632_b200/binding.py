@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.cat_loss_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 10 + [vp, sz, vp]
         L.cat_loss_fwd_static.restype = ctypes.c_int
         L.cat_loss_fwd_static.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 10 + [vp]
+        L.cat_loss_fwd_bwd.restype = ctypes.c_int
+        L.cat_loss_fwd_bwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 13 + [ctypes.c_int, vp, sz, vp]
         L.cat_loss_bwd.restype = ctypes.c_int
         L.cat_loss_bwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 9 + [ctypes.c_int, vp, sz, vp]
         _lib = L
@@ -114,6 +116,16 @@ def cat_loss_bwd(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, acc
                             _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_loss_bwd")
+
+
+def cat_loss_fwd_bwd(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW,
+                     accumulate_dW, workspace) -> None:
+    rc = lib().cat_loss_fwd_bwd(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(conf_ext),
+                                _ptr(grad_loss), _ptr(loss), _ptr(lse), _ptr(conf), _ptr(weight), _ptr(stats),
+                                _ptr(dH), _ptr(dW), int(bool(accumulate_dW)), _ptr(workspace),
+                                workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_loss_fwd_bwd")
 
 
 def read_stats(stats_tensor: torch.Tensor) -> cat_stats:

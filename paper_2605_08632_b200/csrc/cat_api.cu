@@ -23,6 +23,7 @@ constexpr size_t kHeaderBytes = 256;     // workspace header: int32 status at by
 constexpr size_t kScaleOffset = 64;
 constexpr int kMaxSplits = 128;
 constexpr long long kDefaultSlabMiB = 2048;
+constexpr long long kDefaultFusedSlabMiB = 2560;
 
 inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 inline long long cdiv(long long a, long long b) { return (a + b - 1) / b; }
@@ -107,6 +108,82 @@ BwdPlan plan_bwd(const cat_shape* s) {
     p.off_dz = off; off = align256(off + elt * static_cast<size_t>(s->T) * p.Vs);
     p.off_dh_acc = off;
     if (s->in_dtype == CAT_BF16 && p.n_slabs > 1) off = align256(off + sizeof(float) * static_cast<size_t>(s->T) * s->d);
+    p.total = off;
+    return p;
+}
+
+// Fused forward+backward: rows are processed in slabs of whole 128-row tiles and whole draft
+// blocks; one slab of fp16 logits (turned into bf16 dz in place) is the only large scratch.
+struct FusedPlan {
+    long long Ts;          // rows per slab (multiple of lcm(K, 128)), last slab may be shorter
+    long long ldz;         // row pitch of the logits slab (V rounded up to 256)
+    int n_slabs;
+    int S_max;             // largest vocabulary split count over the slabs
+    int n_row_ctas;        // per-row / per-block kernel CTAs summed over the slabs
+    bool warp_scan;
+    bool dw_acc;           // bf16 dW with several slabs: accumulate in an fp32 scratch copy
+    size_t off_part_m, off_part_l, off_z_label, off_row_ce, off_partials, off_z, off_dw_acc, total;
+};
+
+int fwd_splits(long long rows, long long V) {
+    const long long num_m = cdiv(rows, tc::BM), num_n = cdiv(V, tc::BN);
+    const long long smax = num_n < kMaxSplits ? num_n : kMaxSplits;
+    double best = 1e300;
+    int S_best = 1;
+    for (long long S = 1; S <= smax; ++S) {
+        const double cost = static_cast<double>(cdiv(num_m * S, kPlanSMs)) * static_cast<double>(cdiv(num_n, S)) + 1e-3 * S;
+        if (cost < best) { best = cost; S_best = static_cast<int>(S); }
+    }
+    return S_best;
+}
+
+long long gcd_ll(long long a, long long b) { return b == 0 ? a : gcd_ll(b, a % b); }
+
+FusedPlan plan_fused(const cat_shape* s) {
+    FusedPlan p;
+    p.ldz = cdiv(s->V, 256) * 256;
+    const long long L = (static_cast<long long>(s->K) * tc::BM) / gcd_ll(s->K, tc::BM);   // lcm(K, 128)
+    const long long mib = s->slab_mib > 0 ? s->slab_mib : kDefaultFusedSlabMiB;
+    long long cap = ((mib << 20) / (p.ldz * 2) / L) * L;       // rows that fit the slab budget
+    const long long most = ((s->T - 1) / L) * L;                // at least two slabs: the T x V logits never coexist
+    if (most >= L && cap > most) cap = most;
+    if (cap < L) cap = L;
+    // among slab heights within the budget, take the one with the fewest waves of dH tiles
+    // (tiles per slab = rows/128 * d/256, run 148 at a time), then the fewest slabs
+    const long long n_tiles_n = cdiv(s->d, tc::BN);
+    long long best_ts = cap;
+    long long best_waves = -1, best_slabs = 0;
+    for (long long ts = cap, tries = 0; ts >= L && tries < 96; ts -= L, ++tries) {
+        long long waves = 0, slabs = 0;
+        for (long long r0 = 0; r0 < s->T; r0 += ts, ++slabs) {
+            const long long rws = (s->T - r0) < ts ? (s->T - r0) : ts;
+            waves += cdiv(cdiv(rws, tc::BM) * n_tiles_n, kPlanSMs);
+        }
+        if (best_waves < 0 || waves < best_waves || (waves == best_waves && slabs < best_slabs)) {
+            best_waves = waves; best_slabs = slabs; best_ts = ts;
+        }
+    }
+    p.Ts = best_ts;
+    p.n_slabs = static_cast<int>(cdiv(s->T, p.Ts));
+    p.warp_scan = s->K <= 32 && (s->K & (s->K - 1)) == 0;
+    p.S_max = 1;
+    p.n_row_ctas = 0;
+    for (long long r0 = 0; r0 < s->T; r0 += p.Ts) {
+        const long long rws = (s->T - r0) < p.Ts ? (s->T - r0) : p.Ts;
+        const int S = fwd_splits(rws, s->V);
+        if (S > p.S_max) p.S_max = S;
+        p.n_row_ctas += static_cast<int>(cdiv(p.warp_scan ? rws : rws / s->K, rows::ROW_THREADS));
+    }
+    p.dw_acc = s->dW_dtype == CAT_BF16 && p.n_slabs > 1;
+    size_t off = kHeaderBytes;
+    p.off_part_m = off;  off = align256(off + sizeof(float) * p.S_max * s->T);
+    p.off_part_l = off;  off = align256(off + sizeof(float) * p.S_max * s->T);
+    p.off_z_label = off; off = align256(off + sizeof(float) * s->T);
+    p.off_row_ce = off;  off = align256(off + sizeof(float) * s->T);
+    p.off_partials = off; off = align256(off + sizeof(rows::CtaPartial) * p.n_row_ctas);
+    p.off_z = off;       off = align256(off + 2 * static_cast<size_t>(p.Ts) * p.ldz);
+    p.off_dw_acc = off;
+    if (p.dw_acc) off = align256(off + sizeof(float) * static_cast<size_t>(s->V) * s->d);
     p.total = off;
     return p;
 }
@@ -217,6 +294,11 @@ size_t cat_loss_workspace_bytes(const cat_shape* shape, int pass) {
     if (check_shape(shape) != CAT_OK) return 0;
     if (pass == 0) return plan_fwd(shape).total;
     if (pass == 1) return plan_bwd(shape).total;
+    if (pass == 2) {
+        if (shape->in_dtype == CAT_BF16) return plan_fused(shape).total;
+        const size_t a = plan_fwd(shape).total, b = plan_bwd(shape).total;
+        return a > b ? a : b;
+    }
     return 0;
 }
 
@@ -224,6 +306,12 @@ int cat_loss_launch_count(const cat_shape* shape, int pass) {
     if (check_shape(shape) != CAT_OK) return 0;
     if (pass == 0) return 1 + (plan_fwd(shape).warp_scan ? 1 : 2) + 1;
     if (pass == 1) return 1 + 3 * plan_bwd(shape).n_slabs;
+    if (pass == 2) {
+        if (shape->in_dtype != CAT_BF16)
+            return cat_loss_launch_count(shape, 0) + cat_loss_launch_count(shape, 1);
+        const FusedPlan p = plan_fused(shape);
+        return 1 + p.n_slabs * (1 + (p.warp_scan ? 1 : 2) + 1 + 2) + 1;
+    }
     return 0;
 }
 
@@ -266,6 +354,7 @@ int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int
         tc::EpiFwd::Params ep;
         ep.labels = reinterpret_cast<const long long*>(labels);
         ep.part_m = part_m; ep.part_l = part_l; ep.z_label = z_label; ep.T = T; ep.V = V;
+        ep.zs = nullptr; ep.ldz = 0; ep.part_stride = T;
         const int rc = launch_tc<0, 0, tc::EpiFwd>(tmH, tmW, sched, ep, status, sm_count, st);
         if (rc != CAT_OK) return rc;
     } else {
@@ -286,7 +375,7 @@ int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int
     rp.part_m = part_m; rp.part_l = part_l; rp.z_label = z_label;
     rp.labels = reinterpret_cast<const long long*>(labels); rp.valid = valid; rp.conf_ext = conf_ext;
     rp.lse = lse; rp.conf = conf; rp.weight = weight; rp.row_ce = row_ce; rp.partials = partials;
-    rp.T = T; rp.V = V; rp.K = shape->K; rp.S = plan.S;
+    rp.T = T; rp.V = V; rp.K = shape->K; rp.S = plan.S; rp.part_stride = T;
     if (plan.warp_scan) {
         rows::row_kernel<true><<<plan.n_row_ctas, rows::ROW_THREADS, 0, st>>>(rp);
     } else {
@@ -421,6 +510,137 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
         }
     }
     return CAT_OK;
+}
+
+int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                     const float* conf_ext, const float* grad_loss, float* loss, float* lse, float* conf, float* weight,
+                     cat_stats* stats, void* dH, void* dW, int accumulate_dW, void* workspace, size_t workspace_bytes,
+                     void* cuda_stream) {
+    if (!shape || !H || !W || !labels || !loss || !lse || !conf || !weight || !dH || !dW) return CAT_ERR_NULL;
+    const int sc = check_shape(shape);
+    if (sc != CAT_OK) return sc;
+    if (shape->in_dtype != CAT_BF16) {
+        // fp32 path: forward then backward, sharing one workspace (the passes run back to back)
+        const size_t need = cat_loss_workspace_bytes(shape, 2);
+        if (!workspace || misaligned(workspace, 256) || workspace_bytes < need) return CAT_ERR_WORKSPACE;
+        const int rc = cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, workspace,
+                                    workspace_bytes, cuda_stream);
+        if (rc != CAT_OK) return rc;
+        return cat_loss_bwd(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace,
+                            workspace_bytes, cuda_stream);
+    }
+    if (misaligned(H, 16) || misaligned(W, 16) || misaligned(dH, 16) || misaligned(dW, 16) || misaligned(labels, 8) ||
+        misaligned(loss, 4) || misaligned(lse, 4) || misaligned(conf, 4) || misaligned(weight, 4) ||
+        (conf_ext && misaligned(conf_ext, 4)) || (grad_loss && misaligned(grad_loss, 4)) || (stats && misaligned(stats, 8)))
+        return CAT_ERR_ALIGN;
+    const FusedPlan plan = plan_fused(shape);
+    if (!workspace || misaligned(workspace, 256) || workspace_bytes < plan.total) return CAT_ERR_WORKSPACE;
+    int sm_count = 0;
+    const int dc = check_device(&sm_count);
+    if (dc != CAT_OK) return dc;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws);
+    float* scale = reinterpret_cast<float*>(ws + kScaleOffset);
+    float* part_m = reinterpret_cast<float*>(ws + plan.off_part_m);
+    float* part_l = reinterpret_cast<float*>(ws + plan.off_part_l);
+    float* z_label = reinterpret_cast<float*>(ws + plan.off_z_label);
+    float* row_ce = reinterpret_cast<float*>(ws + plan.off_row_ce);
+    rows::CtaPartial* partials = reinterpret_cast<rows::CtaPartial*>(ws + plan.off_partials);
+    void* zs = ws + plan.off_z;
+    float* dw_acc = reinterpret_cast<float*>(ws + plan.off_dw_acc);
+    const int T = static_cast<int>(shape->T), V = static_cast<int>(shape->V), d = static_cast<int>(shape->d);
+    const long long* y = reinterpret_cast<const long long*>(labels);
+    const __nv_bfloat16* Hb = static_cast<const __nv_bfloat16*>(H);
+
+    CUtensorMap tmW_k, tmW_mn;
+    if (tmap_k_major(&tmW_k, W, shape->V, shape->d, shape->ldW, tc::BN) != CAT_OK) return CAT_ERR_CUDA;
+    if (tmap_mn_major(&tmW_mn, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    rows::bwd_scale_kernel<<<1, 1024, 0, st>>>(y, valid, T, V, grad_loss, scale);
+    if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+
+    int cta0 = 0;
+    for (int sl = 0; sl < plan.n_slabs; ++sl) {
+        const long long r0 = static_cast<long long>(sl) * plan.Ts;
+        const long long rws = (shape->T - r0) < plan.Ts ? (shape->T - r0) : plan.Ts;
+        const bool first = sl == 0, last = sl == plan.n_slabs - 1;
+        const int S = fwd_splits(rws, shape->V);
+        const __nv_bfloat16* Hs = Hb + r0 * shape->ldH;
+        CUtensorMap tmH_k, tmH_mn, tmZ_k, tmZ_mn;
+        if (tmap_k_major(&tmH_k, Hs, rws, shape->d, shape->ldH, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_mn_major(&tmH_mn, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_k_major(&tmZ_k, zs, rws, shape->V, plan.ldz, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_mn_major(&tmZ_mn, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
+        {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
+            const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);
+            tc::EpiFwdStore::Params ep;
+            ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
+            ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T;
+            ep.T = static_cast<int>(rws); ep.V = V;
+            const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        }
+        int n_ctas;
+        {   // lse, confidence (Eq. 9), CAT weights (Eq. 10), loss partials of the slab's blocks
+            rows::RowParams rp;
+            rp.part_m = part_m + r0; rp.part_l = part_l + r0; rp.z_label = z_label + r0; rp.labels = y + r0;
+            rp.valid = valid ? valid + r0 : nullptr; rp.conf_ext = conf_ext ? conf_ext + r0 : nullptr;
+            rp.lse = lse + r0; rp.conf = conf + r0; rp.weight = weight + r0; rp.row_ce = row_ce + r0;
+            rp.partials = partials + cta0; rp.part_stride = T;
+            rp.T = static_cast<int>(rws); rp.V = V; rp.K = shape->K; rp.S = S;
+            if (plan.warp_scan) {
+                n_ctas = static_cast<int>(cdiv(rws, rows::ROW_THREADS));
+                rows::row_kernel<true><<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
+            } else {
+                n_ctas = static_cast<int>(cdiv(rws / shape->K, rows::ROW_THREADS));
+                rows::row_kernel<false><<<static_cast<unsigned>(cdiv(rws, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(rp);
+                rows::block_scan_kernel<<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
+            }
+            cta0 += n_ctas;
+        }
+        // logits -> dz in place
+        rows::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
+            zs, plan.ldz, y + r0, valid ? valid + r0 : nullptr, lse + r0, weight + r0, z_label + r0, V);
+        if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+        {   // dH[r0 : r0 + rws, :] = (g/N) dz W : the whole vocabulary is contracted, written once
+            const tc::Sched sched = make_sched(rws, shape->d, shape->V, 0, 1, 1);
+            tc::EpiOut::Params ep;
+            memset(&ep, 0, sizeof(ep));
+            ep.alpha = scale; ep.M = static_cast<int>(rws); ep.N = d;
+            ep.out_bf16 = static_cast<__nv_bfloat16*>(dH) + r0 * shape->ldH; ep.ld_out = shape->ldH;
+            const int rc = launch_tc<0, 1, tc::EpiOut>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        }
+        {   // dW += (g/N) dz^T H[r0 : r0 + rws, :]
+            const tc::Sched sched = make_sched(shape->V, shape->d, rws, 0, 1, 1);
+            tc::EpiOut::Params ep;
+            memset(&ep, 0, sizeof(ep));
+            ep.alpha = scale; ep.M = V; ep.N = d;
+            if (shape->dW_dtype == CAT_F32) {
+                ep.out_f32 = static_cast<float*>(dW); ep.ld_out = shape->ldW;
+                if (!first || accumulate_dW) { ep.add_f32 = ep.out_f32; ep.ld_add = shape->ldW; }
+            } else if (!plan.dw_acc) {
+                ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW;
+                if (accumulate_dW) { ep.add_bf16 = ep.out_bf16; ep.ld_add = shape->ldW; }
+            } else {
+                // bf16 dW over several slabs: sum in fp32 scratch, round once at the end
+                if (first) {
+                    if (accumulate_dW) { ep.add_bf16 = static_cast<const __nv_bfloat16*>(dW); ep.ld_add = shape->ldW; }
+                } else {
+                    ep.add_f32 = dw_acc; ep.ld_add = shape->d;
+                }
+                if (last) { ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW; }
+                else { ep.out_f32 = dw_acc; ep.ld_out = shape->d; }
+            }
+            const int rc = launch_tc<1, 1, tc::EpiOut>(tmZ_mn, tmH_mn, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        }
+    }
+    rows::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(partials, cta0, T / shape->K, loss,
+                                                         reinterpret_cast<rows::StatsOut*>(stats), status);
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------

@@ -5,6 +5,8 @@
 // These touch O(T) data and are bandwidth/latency-bound; no tensor cores are involved.
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace cat {
@@ -22,8 +24,8 @@ struct CtaPartial {
 };
 
 struct RowParams {
-    const float* part_m;       // [S][T]
-    const float* part_l;       // [S][T]
+    const float* part_m;       // [S][part_stride]
+    const float* part_l;       // [S][part_stride]
     const float* z_label;      // [T]
     const long long* labels;   // [T]
     const unsigned char* valid;  // [T] or nullptr
@@ -33,6 +35,7 @@ struct RowParams {
     float* weight;             // [T]
     float* row_ce;             // [T] scratch: lse - z_label (0 for invalid rows); used by the general-K path
     CtaPartial* partials;      // [gridDim.x]
+    long long part_stride;     // row pitch of the partial arrays (>= T)
     int T, V, K, S;
 };
 
@@ -73,10 +76,10 @@ __global__ void __launch_bounds__(ROW_THREADS) row_kernel(const RowParams p) {
     if (in_range) {
         // merge the per-split (max, sum-exp) pairs in split order
         float m = -INFINITY;
-        for (int s = 0; s < p.S; ++s) m = fmaxf(m, p.part_m[static_cast<size_t>(s) * p.T + r]);
+        for (int s = 0; s < p.S; ++s) m = fmaxf(m, p.part_m[static_cast<size_t>(s) * p.part_stride + r]);
         float l = 0.f;
         for (int s = 0; s < p.S; ++s)
-            l += p.part_l[static_cast<size_t>(s) * p.T + r] * expf(p.part_m[static_cast<size_t>(s) * p.T + r] - m);
+            l += p.part_l[static_cast<size_t>(s) * p.part_stride + r] * expf(p.part_m[static_cast<size_t>(s) * p.part_stride + r] - m);
         const float lse = m + logf(l);
         p.lse[r] = lse;
         const long long y = p.labels[r];
@@ -196,6 +199,53 @@ __global__ void __launch_bounds__(1024) bwd_scale_kernel(const long long* labels
         for (int w = 0; w < 32; ++w) tot += sh[w];
         const float g = grad_loss ? *grad_loss : 1.f;
         *scale = tot > 0 ? g / static_cast<float>(tot) : 0.f;
+    }
+}
+
+// Fused path: turn one row of stored fp16 logits into bf16 dz in place,
+//   dz[r, v] = weight_r * (exp(z[r, v] - lse_r) - [v == y_r]),
+// the label entry formed from the fp32 label logit.  One CTA per row, 16-byte vectors; columns
+// at or beyond V are written as zero.  Pure streaming: 2 bytes read + 2 bytes written per logit.
+__global__ void __launch_bounds__(ROW_THREADS) z_to_dz_kernel(void* zs, long long ldz, const long long* labels,
+                                                              const unsigned char* valid, const float* lse,
+                                                              const float* weight, const float* z_label, int V) {
+    const int r = blockIdx.x;
+    const long long y = labels[r];
+    const bool ok = (valid == nullptr || valid[r] != 0) && y >= 0 && y < V;
+    const float w = ok ? weight[r] : 0.f;
+    const float l2 = ok ? lse[r] * 1.4426950408889634f : INFINITY;
+    const int yi = ok ? static_cast<int>(y) : -1;
+    const float dz_label = ok ? w * (expf(z_label[r] - lse[r]) - 1.f) : 0.f;
+    uint4* row = reinterpret_cast<uint4*>(static_cast<unsigned short*>(zs) + static_cast<size_t>(r) * ldz);
+    const int groups = static_cast<int>(ldz / 8);
+    for (int gi = threadIdx.x; gi < groups; gi += ROW_THREADS) {
+        const uint4 in = __ldcs(row + gi);
+        const uint32_t wds[4] = {in.x, in.y, in.z, in.w};
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&wds[i]));
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
+        const int col = gi * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float pz;
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pz) : "f"(fmaf(f[i], 1.4426950408889634f, -l2)));
+            f[i] = (col + i < V) ? w * pz : 0.f;
+            if (col + i == yi) f[i] = dz_label;
+        }
+        uint4 out;
+        __nv_bfloat162 b0 = __floats2bfloat162_rn(f[0], f[1]);
+        __nv_bfloat162 b1 = __floats2bfloat162_rn(f[2], f[3]);
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(f[4], f[5]);
+        __nv_bfloat162 b3 = __floats2bfloat162_rn(f[6], f[7]);
+        out.x = *reinterpret_cast<uint32_t*>(&b0);
+        out.y = *reinterpret_cast<uint32_t*>(&b1);
+        out.z = *reinterpret_cast<uint32_t*>(&b2);
+        out.w = *reinterpret_cast<uint32_t*>(&b3);
+        row[gi] = out;
     }
 }
 

@@ -18,6 +18,7 @@
 #pragma once
 #include "ptx.cuh"
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 namespace cat {
 namespace tc {
@@ -103,12 +104,18 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
 
 // Forward: online max / sum-exp over the vocabulary (softmax partition function of Eq. 11's
 // log P), and the label logit z[r, y_r] picked from the accumulator chunk that holds it.
-struct EpiFwd {
+// STORE = true additionally writes the logits of the tile as fp16 (saturating) into a row slab,
+// for the fused forward+backward path that keeps one slab of logits instead of recomputing them.
+template <bool STORE>
+struct EpiFwdT {
     struct Params {
         const long long* labels;   // [T]
-        float* part_m;             // [n_groups][T] running max of each (row, vocabulary split)
-        float* part_l;             // [n_groups][T] sum exp(z - max)
+        float* part_m;             // [n_groups][part_stride] running max of each (row, vocabulary split)
+        float* part_l;             // [n_groups][part_stride] sum exp(z - max)
         float* z_label;            // [T]
+        __half* zs;                // [T][ldz] fp16 logits (STORE only)
+        long long ldz;
+        long long part_stride;
         int T;
         int V;
     };
@@ -145,6 +152,20 @@ struct EpiFwd {
                 for (int i = 0; i < 32; ++i)
                     if (i >= live) f[i] = -INFINITY;
             }
+            if (STORE) {
+                if (s.row < p.T) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 pk;
+                        pk.x = ptx::pack_f16x2_sat(f[q * 8 + 0], f[q * 8 + 1]);
+                        pk.y = ptx::pack_f16x2_sat(f[q * 8 + 2], f[q * 8 + 3]);
+                        pk.z = ptx::pack_f16x2_sat(f[q * 8 + 4], f[q * 8 + 5]);
+                        pk.w = ptx::pack_f16x2_sat(f[q * 8 + 6], f[q * 8 + 7]);
+                        __stcs(dst + q, pk);
+                    }
+                }
+            }
             const int rel = s.y - (col0 + c * 32);
             if (rel >= 0 && rel < 32) {
                 float zy = 0.f;
@@ -167,11 +188,13 @@ struct EpiFwd {
     }
     __device__ static __forceinline__ void end_item(const Params& p, const State& s, int group) {
         if (s.row < p.T) {
-            p.part_m[static_cast<size_t>(group) * p.T + s.row] = s.m_run;
-            p.part_l[static_cast<size_t>(group) * p.T + s.row] = s.l_run;
+            p.part_m[static_cast<size_t>(group) * p.part_stride + s.row] = s.m_run;
+            p.part_l[static_cast<size_t>(group) * p.part_stride + s.row] = s.l_run;
         }
     }
 };
+using EpiFwd = EpiFwdT<false>;
+using EpiFwdStore = EpiFwdT<true>;
 
 // Backward recompute: dz[r, v] = weight_r * (exp(z - lse_r) - [v == y_r]) as a bf16 tile of the
 // current vocabulary slab (the scalar g/N is applied later, in fp32, by the dH / dW epilogues).

@@ -48,6 +48,26 @@ def run_gpu(batch, slab_mib=0, g=None, conf_ext=None, dW_dtype=torch.float32, us
     return out
 
 
+def run_gpu_fused(batch, slab_mib=0, g=None, conf_ext=None, dW_dtype=torch.float32, use_valid=True, accumulate_into=None):
+    """Same outputs as run_gpu, through the single cat_loss_fwd_bwd call."""
+    dev = torch.device("cuda")
+    H, W = batch.H.to(dev), batch.W.to(dev)
+    labels = batch.labels.to(dev)
+    valid = batch.valid.to(dev) if use_valid else None
+    cl = CatLoss(batch.T, batch.d, batch.V, batch.K, dtype=batch.torch_dtype, dW_dtype=dW_dtype, slab_mib=slab_mib)
+    ce = None if conf_ext is None else torch.as_tensor(conf_ext, dtype=torch.float32, device=dev)
+    gl = None if g is None else torch.tensor([g], dtype=torch.float32, device=dev)
+    acc = False
+    if accumulate_into is not None:
+        cl.dW.copy_(torch.as_tensor(accumulate_into, device=dev).to(dW_dtype))
+        acc = True
+    cl.forward_backward(H, W, labels, valid, ce, gl, accumulate_dW=acc)
+    torch.cuda.synchronize()
+    return dict(loss=float(cl.loss.item()), lse=cl.lse.cpu().numpy(), conf=cl.conf.cpu().numpy(),
+                weight=cl.weight.cpu().numpy(), dH=cl.dH.float().cpu().numpy(), dW=cl.dW.float().cpu().numpy(),
+                stats=cl.fwd_stats(), bwd_status=cl.fused_status(), obj=cl)
+
+
 def run_oracle(batch, g=1.0, conf_ext=None, use_valid=True):
     fwd, dH, dW = O.cat_forward_backward(batch.H, batch.W, batch.labels, batch.valid if use_valid else None, batch.K,
                                          conf_ext=conf_ext, g=g)

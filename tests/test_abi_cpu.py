@@ -51,7 +51,12 @@ def test_workspace_sizes():
     assert B.cat_loss_workspace_bytes(big, 1) < 0.15 * (131072 * 128256 * 2)
     capped = B.make_shape(16384, 2048, 128256, 8, B.CAT_BF16, slab_mib=256)
     assert B.cat_loss_workspace_bytes(capped, 1) < (256 << 20) + 16384 * 2048 * 4 + (1 << 20)
-    assert B.cat_loss_workspace_bytes(s, 2) == 0
+    fused = B.cat_loss_workspace_bytes(s, 2)
+    assert 0 < fused < 0.62 * logits_bytes        # one slab of logits, at least two slabs per batch
+    assert B.cat_loss_workspace_bytes(big, 2) < 0.1 * (131072 * 128256 * 2)
+    assert B.cat_loss_workspace_bytes(s, 3) == 0
+    assert B.cat_loss_launch_count(s, 0) == 3 and B.cat_loss_launch_count(s, 1) == 7
+    assert B.cat_loss_launch_count(s, 2) == 1 + 2 * 5 + 1
 
 
 @pytest.mark.parametrize("kw,code", [

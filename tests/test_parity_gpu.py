@@ -10,7 +10,7 @@ from paper_2605_08632_b200 import synth
 from paper_2605_08632_b200 import binding as B
 from paper_2605_08632_b200.api import CatLoss
 
-from parity_util import TOL, check_backward, check_forward, rel_l2, run_gpu, run_oracle
+from parity_util import TOL, check_backward, check_forward, rel_l2, run_gpu, run_gpu_fused, run_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -127,6 +127,50 @@ def test_row_pitch_larger_than_d():
     assert rel_l2(cl.dH[:, :192].float().cpu().numpy(), dH) <= 1e-2
     assert rel_l2(cl.dW[:, :192].cpu().numpy(), dW) <= 1e-2
     assert torch.all(cl.dH[:, 192:] == 3.0) and torch.all(cl.dW[:, 192:] == 3.0)
+
+
+# ---------------------------------------------------------------- fused forward+backward (no recompute)
+def _fused_check(batch, **kw):
+    gpu = run_gpu_fused(batch, **kw)
+    fwd, dH, dW = run_oracle(batch, g=kw.get("g") or 1.0, conf_ext=kw.get("conf_ext"), use_valid=kw.get("use_valid", True))
+    check_forward(gpu, fwd, batch.K, batch.torch_dtype, batch.V)
+    check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype)
+    return gpu, fwd
+
+
+@pytest.mark.parametrize("cfg,T", [(2, 600), (3, 400), (41, 520), (5, 448)])
+def test_fused_reduced_configs_full_d_V_K(cfg, T):
+    batch = synth.make_batch(cfg, T=T - T % synth.CONFIGS[cfg].K)
+    _fused_check(batch)
+
+
+def test_fused_many_row_slabs_ragged_shapes_and_options():
+    batch = synth.make_batch(41, T=1000, d=200, V=5003 - 3, K=8)      # 8 slabs of 128 rows, ragged last slab
+    gpu, fwd = _fused_check(batch, slab_mib=1, g=0.1)
+    assert B.cat_loss_launch_count(gpu["obj"].shape, 2) == 1 + 8 * 5 + 1
+    rng = np.random.default_rng(7)
+    _fused_check(batch, slab_mib=2, conf_ext=rng.random(1000).astype(np.float32), use_valid=False)
+    _, dH, dW = run_oracle(batch)
+    base = rng.standard_normal(dW.shape).astype(np.float32) * float(np.abs(dW).max())
+    acc = run_gpu_fused(batch, slab_mib=1, accumulate_into=base)
+    assert rel_l2(acc["dW"], dW + base) <= 1e-4
+    bf = run_gpu_fused(batch, slab_mib=1, dW_dtype=torch.bfloat16)    # fp32 scratch accumulation, rounded once
+    assert rel_l2(bf["dW"], dW) <= 1.2e-2
+
+
+@pytest.mark.parametrize("K", [1, 3, 40])
+def test_fused_block_lengths(K):
+    batch = synth.make_batch(41, T=K * 24, d=128, V=1024, K=K)
+    _fused_check(batch, slab_mib=1)
+
+
+def test_fused_fp32_inputs_and_determinism():
+    batch = synth.make_batch(1)
+    _fused_check(batch)
+    b2 = synth.make_batch(2, T=512, V=20000)
+    a, b = run_gpu_fused(b2, slab_mib=8), run_gpu_fused(b2, slab_mib=8)
+    for key in ("lse", "conf", "weight", "dH", "dW"):
+        assert a[key].tobytes() == b[key].tobytes(), key
 
 
 def test_errors_on_gpu_box_leave_context_usable():
