@@ -112,6 +112,8 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override T (debug / profiling of a small case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", choices=["fused", "two-call"], default=None,
+                    help="run only that path for --warmup + --steps steps and exit (for ncu captures of a small case; prints no bench line)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -184,6 +186,13 @@ def main():
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             return float(t.item())
         return ms
+
+    if args.profile:
+        for _ in range(args.warmup + args.steps):
+            step() if args.profile == "fused" else step_split()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_run": args.profile, "T": T, "note": "not a benchmark value"}))
+        return
 
     stream = torch.cuda.current_stream()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
