@@ -8,6 +8,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <stdlib.h>
+
 #include <mutex>
 
 #include "rowops.cuh"
@@ -27,6 +29,19 @@ constexpr long long kDefaultFusedSlabMiB = 2560;
 
 inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 inline long long cdiv(long long a, long long b) { return (a + b - 1) / b; }
+
+// CTAs per tensor-core output tile: 2 (a CTA pair shares a 256 x 256 tile, tcgen05 cta_group::2)
+// unless the environment variable CAT_LOSS_CTA_PAIR=0 selects the one-CTA 128 x 256 kernel.
+// Read once per process: plans and workspace sizes depend on it.
+int cta_group() {
+    static const int cg = [] {
+        const char* e = getenv("CAT_LOSS_CTA_PAIR");
+        return (e && e[0] == '0') ? 1 : 2;
+    }();
+    return cg;
+}
+inline long long tile_m() { return static_cast<long long>(tc::BM) * cta_group(); }   // rows per scheduled m-tile
+inline long long plan_workers() { return kPlanSMs / cta_group(); }                    // CTAs or CTA pairs
 
 // ------------------------------------------------------------------------------ validation
 int check_shape(const cat_shape* s) {
@@ -53,18 +68,24 @@ struct FwdPlan {
     size_t off_part_m, off_part_l, off_z_label, off_row_ce, off_partials, total;
 };
 
+// Vocabulary splits of the forward GEMM: persistent workers (CTAs or CTA pairs) take items
+// (m-tile, split) round-robin, so the cost is waves * longest item, plus a small charge per split.
+int fwd_splits(long long rows, long long V) {
+    const long long num_m = cdiv(rows, tile_m()), num_n = cdiv(V, tc::BN);
+    const long long smax = num_n < kMaxSplits ? num_n : kMaxSplits;
+    double best = 1e300;
+    int S_best = 1;
+    for (long long S = 1; S <= smax; ++S) {
+        const double cost = static_cast<double>(cdiv(num_m * S, plan_workers())) * static_cast<double>(cdiv(num_n, S)) + 1e-3 * S;
+        if (cost < best) { best = cost; S_best = static_cast<int>(S); }
+    }
+    return S_best;
+}
+
 FwdPlan plan_fwd(const cat_shape* s) {
     FwdPlan p;
     if (s->in_dtype == CAT_BF16) {
-        const long long num_m = cdiv(s->T, tc::BM), num_n = cdiv(s->V, tc::BN);
-        const long long smax = num_n < kMaxSplits ? num_n : kMaxSplits;
-        double best = 1e300;
-        p.S = 1;
-        for (long long S = 1; S <= smax; ++S) {
-            // persistent CTAs take items round-robin: waves * longest item, plus a small charge per split
-            const double cost = static_cast<double>(cdiv(num_m * S, kPlanSMs)) * static_cast<double>(cdiv(num_n, S)) + 1e-3 * S;
-            if (cost < best) { best = cost; p.S = static_cast<int>(S); }
-        }
+        p.S = fwd_splits(s->T, s->V);
     } else {
         const long long num_m = cdiv(s->T, simt::TM), num_n = cdiv(s->V, simt::TN);
         long long S = (2 * kPlanSMs) / num_m;
@@ -112,10 +133,10 @@ BwdPlan plan_bwd(const cat_shape* s) {
     return p;
 }
 
-// Fused forward+backward: rows are processed in slabs of whole 128-row tiles and whole draft
+// Fused forward+backward: rows are processed in slabs of whole m-tiles and whole draft
 // blocks; one slab of fp16 logits (turned into bf16 dz in place) is the only large scratch.
 struct FusedPlan {
-    long long Ts;          // rows per slab (multiple of lcm(K, 128)), last slab may be shorter
+    long long Ts;          // rows per slab (multiple of lcm(K, rows per m-tile)), last slab may be shorter
     long long ldz;         // row pitch of the logits slab (V rounded up to 256)
     int n_slabs;
     int S_max;             // largest vocabulary split count over the slabs
@@ -125,31 +146,19 @@ struct FusedPlan {
     size_t off_part_m, off_part_l, off_z_label, off_row_ce, off_partials, off_z, off_dw_acc, total;
 };
 
-int fwd_splits(long long rows, long long V) {
-    const long long num_m = cdiv(rows, tc::BM), num_n = cdiv(V, tc::BN);
-    const long long smax = num_n < kMaxSplits ? num_n : kMaxSplits;
-    double best = 1e300;
-    int S_best = 1;
-    for (long long S = 1; S <= smax; ++S) {
-        const double cost = static_cast<double>(cdiv(num_m * S, kPlanSMs)) * static_cast<double>(cdiv(num_n, S)) + 1e-3 * S;
-        if (cost < best) { best = cost; S_best = static_cast<int>(S); }
-    }
-    return S_best;
-}
-
 long long gcd_ll(long long a, long long b) { return b == 0 ? a : gcd_ll(b, a % b); }
 
 FusedPlan plan_fused(const cat_shape* s) {
     FusedPlan p;
     p.ldz = cdiv(s->V, 256) * 256;
-    const long long L = (static_cast<long long>(s->K) * tc::BM) / gcd_ll(s->K, tc::BM);   // lcm(K, 128)
+    const long long L = (static_cast<long long>(s->K) * tile_m()) / gcd_ll(s->K, tile_m());   // lcm(K, rows per m-tile)
     const long long mib = s->slab_mib > 0 ? s->slab_mib : kDefaultFusedSlabMiB;
     long long cap = ((mib << 20) / (p.ldz * 2) / L) * L;       // rows that fit the slab budget
     const long long most = ((s->T - 1) / L) * L;                // at least two slabs: the T x V logits never coexist
     if (most >= L && cap > most) cap = most;
     if (cap < L) cap = L;
     // among slab heights within the budget, take the one with the fewest waves of dH tiles
-    // (tiles per slab = rows/128 * d/256, run 148 at a time), then the fewest slabs
+    // (tiles per slab = m-tiles * d/256, one per worker at a time), then the fewest slabs
     const long long n_tiles_n = cdiv(s->d, tc::BN);
     long long best_ts = cap;
     long long best_waves = -1, best_slabs = 0;
@@ -157,7 +166,7 @@ FusedPlan plan_fused(const cat_shape* s) {
         long long waves = 0, slabs = 0;
         for (long long r0 = 0; r0 < s->T; r0 += ts, ++slabs) {
             const long long rws = (s->T - r0) < ts ? (s->T - r0) : ts;
-            waves += cdiv(cdiv(rws, tc::BM) * n_tiles_n, kPlanSMs);
+            waves += cdiv(cdiv(rws, tile_m()) * n_tiles_n, plan_workers());
         }
         if (best_waves < 0 || waves < best_waves || (waves == best_waves && slabs < best_slabs)) {
             best_waves = waves; best_slabs = slabs; best_ts = ts;
@@ -239,27 +248,61 @@ inline int tmap_mn_major(CUtensorMap* m, const void* base, long long k, long lon
     return make_tmap(m, base, k, mn, ld, 64, tc::BK);              // [K rows][MN cols]
 }
 
+// K-major A operand: this CTA's 128 rows.  K-major B operand: the 256 columns of the tile, or the
+// 128 of them that one CTA of a pair loads.
+inline int tmap_a(CUtensorMap* m, const void* base, long long mn, long long k, long long ld) {
+    return tmap_k_major(m, base, mn, k, ld, tc::BM);
+}
+inline int tmap_b(CUtensorMap* m, const void* base, long long mn, long long k, long long ld) {
+    return tmap_k_major(m, base, mn, k, ld, tc::BN / cta_group());
+}
+
 int band_tiles(long long d) {
-    long long b = (64ll << 20) / (tc::BM * d * 2);
+    long long b = (64ll << 20) / (tile_m() * d * 2);
     return static_cast<int>(b < 1 ? 1 : b);
+}
+
+template <int A_MN, int B_MN, class Epi, int CG>
+int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& sched, const typename Epi::Params& ep,
+                 int* status, int sm_count, cudaStream_t st) {
+    auto kern = tc::gemm_kernel<A_MN, B_MN, Epi, CG>;
+    constexpr int smem = tc::Geo<CG>::SMEM_BYTES;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return CAT_ERR_CUDA;
+    }
+    const int workers = sm_count / CG;
+    const int grid = CG * (sched.n_items < workers ? sched.n_items : workers);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(tc::NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tmA, tmB, sched, ep, status) != cudaSuccess) {
+        cudaGetLastError();
+        return CAT_ERR_CUDA;
+    }
+    return CAT_OK;
 }
 
 template <int A_MN, int B_MN, class Epi>
 int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& sched, const typename Epi::Params& ep,
               int* status, int sm_count, cudaStream_t st) {
-    auto kern = tc::gemm_kernel<A_MN, B_MN, Epi>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) {
-        cudaGetLastError();
-        return CAT_ERR_CUDA;
-    }
-    const int grid = sched.n_items < sm_count ? sched.n_items : sm_count;
-    kern<<<grid, tc::NUM_THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, sched, ep, status);
-    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+    return cta_group() == 2 ? launch_tc_cg<A_MN, B_MN, Epi, 2>(tmA, tmB, sched, ep, status, sm_count, st)
+                            : launch_tc_cg<A_MN, B_MN, Epi, 1>(tmA, tmB, sched, ep, status, sm_count, st);
 }
 
 tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int band_m, int n_fastest) {
     tc::Sched s;
-    s.num_m_tiles = static_cast<int>(cdiv(M, tc::BM));
+    s.num_m_tiles = static_cast<int>(cdiv(M, tile_m()));
     s.num_n_tiles = static_cast<int>(cdiv(N, tc::BN));
     s.num_kb = static_cast<int>(cdiv(Kd, tc::BK));
     s.n_groups = n_groups > 0 ? n_groups : s.num_n_tiles;
@@ -344,8 +387,8 @@ int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int
 
     CUtensorMap tmH, tmW;
     if (bf16) {
-        if (tmap_k_major(&tmH, H, shape->T, shape->d, shape->ldH, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
-        if (tmap_k_major(&tmW, W, shape->V, shape->d, shape->ldW, tc::BN) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_a(&tmH, H, shape->T, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_b(&tmW, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
     }
     if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
 
@@ -414,7 +457,7 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
     // tensor maps that do not depend on the slab
     CUtensorMap tmH_k, tmH_mn;
     if (bf16) {
-        if (tmap_k_major(&tmH_k, H, shape->T, shape->d, shape->ldH, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_a(&tmH_k, H, shape->T, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_mn_major(&tmH_mn, H, shape->T, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
     }
     if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
@@ -430,9 +473,9 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
             __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_dz);
             float* dh_acc = reinterpret_cast<float*>(ws + plan.off_dh_acc);
             CUtensorMap tmW_k, tmW_mn, tmDz_k, tmDz_mn;
-            if (tmap_k_major(&tmW_k, Wb, width, shape->d, shape->ldW, tc::BN) != CAT_OK) return CAT_ERR_CUDA;
+            if (tmap_b(&tmW_k, Wb, width, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
             if (tmap_mn_major(&tmW_mn, Wb, width, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
-            if (tmap_k_major(&tmDz_k, dz, shape->T, width, plan.Vs, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+            if (tmap_a(&tmDz_k, dz, shape->T, width, plan.Vs) != CAT_OK) return CAT_ERR_CUDA;
             if (tmap_mn_major(&tmDz_mn, dz, shape->T, width, plan.Vs) != CAT_OK) return CAT_ERR_CUDA;
             {   // recompute the logits of this slab and turn them into dz
                 const tc::Sched sched = make_sched(shape->T, width, shape->d, 0, band_tiles(shape->d), 0);
@@ -555,7 +598,7 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const
     const __nv_bfloat16* Hb = static_cast<const __nv_bfloat16*>(H);
 
     CUtensorMap tmW_k, tmW_mn;
-    if (tmap_k_major(&tmW_k, W, shape->V, shape->d, shape->ldW, tc::BN) != CAT_OK) return CAT_ERR_CUDA;
+    if (tmap_b(&tmW_k, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
     if (tmap_mn_major(&tmW_mn, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
     if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
     rows::bwd_scale_kernel<<<1, 1024, 0, st>>>(y, valid, T, V, grad_loss, scale);
@@ -569,9 +612,9 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const
         const int S = fwd_splits(rws, shape->V);
         const __nv_bfloat16* Hs = Hb + r0 * shape->ldH;
         CUtensorMap tmH_k, tmH_mn, tmZ_k, tmZ_mn;
-        if (tmap_k_major(&tmH_k, Hs, rws, shape->d, shape->ldH, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_a(&tmH_k, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_mn_major(&tmH_mn, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
-        if (tmap_k_major(&tmZ_k, zs, rws, shape->V, plan.ldz, tc::BM) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_a(&tmZ_k, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_mn_major(&tmZ_mn, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
         {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
             const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);

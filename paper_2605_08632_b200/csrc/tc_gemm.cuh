@@ -26,11 +26,8 @@ namespace tc {
 constexpr int BM = 128;
 constexpr int BN = 256;
 constexpr int BK = 64;
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 8;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
-constexpr int B_STAGE_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int MN_ATOM_BYTES = 64 * BK * 2;                // one 64(MN) x BK box of an MN-major operand
@@ -66,8 +63,8 @@ __device__ __forceinline__ void decode_item(const Sched& s, int item, int& m_til
 }
 
 struct Ctl {
-    unsigned long long full[STAGES];
-    unsigned long long empty[STAGES];
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
     unsigned long long tfull[2];
     unsigned long long tempty[2];
     unsigned long long drain;
@@ -350,42 +347,73 @@ struct EpiOut {
 
 // ------------------------------------------------------------------------------------------
 // The kernel.  tmA / tmB are 2-D tiled tensor maps with 128-byte swizzle:
-//   K-major operand  [rows = M or N][cols = K]: box {BK, BM or BN}, one box per stage;
-//   MN-major operand [rows = K][cols = M or N]: box {64, BK}, BM/64 or BN/64 boxes per stage.
+//   K-major operand  [rows = M or N][cols = K]: box {BK, rows of the tile this CTA loads};
+//   MN-major operand [rows = K][cols = M or N]: box {64, BK}, one box per 64 rows of the tile.
 // Rows/columns past the tensor's extent are zero-filled by TMA, which makes ragged M, N and K
 // contribute exact zeros.
+//
+// CG = 1: one CTA per 128 x 256 output tile.
+// CG = 2: a cluster of two CTAs shares a 256 x 256 output tile (tcgen05 cta_group::2).  CTA
+//   `rank` of the pair loads the A rows of its own 128-row half and half of the B tile (128 of
+//   the 256 columns), so a stage is 32 KB instead of 48 KB per CTA and the ring holds six
+//   stages.  The leader (rank 0) issues every MMA; each CTA's accumulator half (its 128 rows x
+//   256 columns) lives in its own TMEM and is drained by its own epilogue warps.  Barrier
+//   wiring: `full` lives in the leader and counts the bytes of both CTAs' loads; `empty` and
+//   `tfull` are signalled in both CTAs at once by the leader's tcgen05.commit; `tempty` lives in
+//   the leader and collects one arrival per epilogue warp of both CTAs.
 // ------------------------------------------------------------------------------------------
-template <int A_MN, int B_MN, class Epi>
+template <int CG>
+struct Geo {
+    static constexpr int STAGES = CG == 1 ? 4 : 6;
+    static constexpr int BN_CTA = BN / CG;                        // B-tile rows this CTA loads
+    static constexpr int B_BYTES = BN_CTA * BK * 2;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
+    static constexpr int TILE_M = BM * CG;                        // output rows per scheduled m-tile
+};
+
+template <int A_MN, int B_MN, class Epi, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const Sched sched, const typename Epi::Params ep, int* status) {
+    using G = Geo<CG>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ Ctl ctl;
     const uint32_t ring = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
+    const int worker = blockIdx.x / CG;          // a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
+    const int n_workers = gridDim.x / CG;
 
     if (threadIdx.x == 0) {
         ptx::prefetch_tmap(&tmA);
         ptx::prefetch_tmap(&tmB);
-        for (int i = 0; i < STAGES; ++i) {
+        for (int i = 0; i < G::STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctl.full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctl.empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctl.tfull[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctl.tempty[i]), NUM_THREADS - 64);
+            ptx::mbar_init(ptx::smem_u32(&ctl.tempty[i]), CG == 1 ? NUM_THREADS - 64 : 2 * (NUM_THREADS - 64) / 32);
         }
         ptx::mbar_init(ptx::smem_u32(&ctl.drain), 1);
         ctl.abort = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
-        ptx::tmem_alloc<TMEM_COLS>(ptx::smem_u32(&ctl.tmem_base));
-        ptx::tmem_relinquish();
+        if (CG == 1) {
+            ptx::tmem_alloc<TMEM_COLS>(ptx::smem_u32(&ctl.tmem_base));
+            ptx::tmem_relinquish();
+        } else {
+            ptx::tmem_alloc_pair<TMEM_COLS>(ptx::smem_u32(&ctl.tmem_base));
+            ptx::tmem_relinquish_pair();
+        }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CG == 1) __syncthreads();
+    else ptx::cluster_sync_all();     // the peer's barriers must exist before anything signals them
     ptx::tc_fence_after();
     const uint32_t tmem = ctl.tmem_base;
     volatile int* abort = &ctl.abort;
@@ -395,52 +423,78 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, issued = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < sched.n_items && ok; item += gridDim.x) {
+            for (int item = worker; item < sched.n_items && ok; item += n_workers) {
                 int m_tile, group, n_begin, n_end;
                 decode_item(sched, item, m_tile, group, n_begin, n_end);
+                const int m0 = (m_tile * CG + static_cast<int>(rank)) * BM;
                 for (int n = n_begin; n < n_end && ok; ++n) {
+                    const int n0 = n * BN + static_cast<int>(rank) * G::BN_CTA;
                     for (int kb = 0; kb < sched.num_kb; ++kb) {
                         if (!wait_bounded(ptx::smem_u32(&ctl.empty[stage]), phase ^ 1u, abort, status)) { ok = false; break; }
-                        const uint32_t full = ptx::smem_u32(&ctl.full[stage]);
-                        ptx::mbar_arrive_expect_tx(full, STAGE_BYTES);
-                        const uint32_t a_dst = ring + stage * STAGE_BYTES;
+                        const uint32_t full_local = ptx::smem_u32(&ctl.full[stage]);
+                        if (leader) ptx::mbar_arrive_expect_tx(full_local, G::STAGE_BYTES * CG);
+                        const uint32_t a_dst = ring + stage * G::STAGE_BYTES;
                         const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                        if (A_MN) {
+                        if (CG == 1) {
+                            if (A_MN) {
 #pragma unroll
-                            for (int j = 0; j < BM / 64; ++j)
-                                ptx::tma_load_2d(a_dst + j * MN_ATOM_BYTES, &tmA, m_tile * BM + j * 64, kb * BK, full);
-                        } else {
-                            ptx::tma_load_2d(a_dst, &tmA, kb * BK, m_tile * BM, full);
-                        }
-                        if (B_MN) {
+                                for (int j = 0; j < BM / 64; ++j)
+                                    ptx::tma_load_2d(a_dst + j * MN_ATOM_BYTES, &tmA, m0 + j * 64, kb * BK, full_local);
+                            } else {
+                                ptx::tma_load_2d(a_dst, &tmA, kb * BK, m0, full_local);
+                            }
+                            if (B_MN) {
 #pragma unroll
-                            for (int j = 0; j < BN / 64; ++j)
-                                ptx::tma_load_2d(b_dst + j * MN_ATOM_BYTES, &tmB, n * BN + j * 64, kb * BK, full);
+                                for (int j = 0; j < G::BN_CTA / 64; ++j)
+                                    ptx::tma_load_2d(b_dst + j * MN_ATOM_BYTES, &tmB, n0 + j * 64, kb * BK, full_local);
+                            } else {
+                                ptx::tma_load_2d(b_dst, &tmB, kb * BK, n0, full_local);
+                            }
                         } else {
-                            ptx::tma_load_2d(b_dst, &tmB, kb * BK, n * BN, full);
+                            const uint32_t full_lead = ptx::mapa_shared(full_local, 0);   // the leader's barrier
+                            if (A_MN) {
+#pragma unroll
+                                for (int j = 0; j < BM / 64; ++j)
+                                    ptx::tma_load_2d_pair(a_dst + j * MN_ATOM_BYTES, &tmA, m0 + j * 64, kb * BK, full_lead);
+                            } else {
+                                ptx::tma_load_2d_pair(a_dst, &tmA, kb * BK, m0, full_lead);
+                            }
+                            if (B_MN) {
+#pragma unroll
+                                for (int j = 0; j < G::BN_CTA / 64; ++j)
+                                    ptx::tma_load_2d_pair(b_dst + j * MN_ATOM_BYTES, &tmB, n0 + j * 64, kb * BK, full_lead);
+                            } else {
+                                ptx::tma_load_2d_pair(b_dst, &tmB, kb * BK, n0, full_lead);
+                            }
                         }
                         ++issued;
-                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        if (++stage == G::STAGES) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
             if (!ok) {
-                // aborted: let the copies already issued land before the CTA exits
-                const uint32_t back = issued < STAGES ? issued : STAGES;
-                for (uint32_t i = 0; i < back; ++i) {
-                    const uint32_t q = issued - 1 - i;
-                    wait_bounded(ptx::smem_u32(&ctl.full[q % STAGES]), (q / STAGES) & 1u, abort, status, 20000000ull);
+                // aborted: let the copies already issued land before the CTA exits.  The leader can
+                // watch its own `full` barriers; the peer, whose copies signal the leader, just waits.
+                if (leader) {
+                    const uint32_t back = issued < G::STAGES ? issued : G::STAGES;
+                    for (uint32_t i = 0; i < back; ++i) {
+                        const uint32_t q = issued - 1 - i;
+                        wait_bounded(ptx::smem_u32(&ctl.full[q % G::STAGES]), (q / G::STAGES) & 1u, abort, status, 20000000ull);
+                    }
+                } else {
+                    const unsigned long long t0 = ptx::globaltimer_ns();
+                    while (ptx::globaltimer_ns() - t0 < 20000000ull) __nanosleep(1000);
                 }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN, A_MN, B_MN);
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM * CG, BN, A_MN, B_MN);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < sched.n_items && ok; item += gridDim.x) {
+            for (int item = worker; item < sched.n_items && ok; item += n_workers) {
                 int m_tile, group, n_begin, n_end;
                 decode_item(sched, item, m_tile, group, n_begin, n_end);
                 for (int n = n_begin; n < n_end && ok; ++n) {
@@ -450,7 +504,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int kb = 0; kb < sched.num_kb; ++kb) {
                         if (!wait_bounded(ptx::smem_u32(&ctl.full[stage]), phase, abort, status)) { ok = false; break; }
                         ptx::tc_fence_after();
-                        const uint32_t a_base = ring + stage * STAGE_BYTES;
+                        const uint32_t a_base = ring + stage * G::STAGE_BYTES;
                         const uint32_t b_base = a_base + A_STAGE_BYTES;
 #pragma unroll
                         for (int j = 0; j < BK / 16; ++j) {
@@ -460,20 +514,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                                         : ptx::smem_desc_sw128(a_base + j * 32, 16, 1024);
                             const uint64_t bdesc = B_MN ? ptx::smem_desc_sw128(b_base + j * 2048, MN_ATOM_BYTES, 1024)
                                                         : ptx::smem_desc_sw128(b_base + j * 32, 16, 1024);
-                            ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
+                            if (CG == 1) ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
+                            else ptx::umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
                         }
-                        ptx::umma_commit(ptx::smem_u32(&ctl.empty[stage]));   // frees the stage once these MMAs have read it
-                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        // frees the stage (in both CTAs of a pair) once these MMAs have read it
+                        if (CG == 1) ptx::umma_commit(ptx::smem_u32(&ctl.empty[stage]));
+                        else ptx::umma_commit_pair(ptx::smem_u32(&ctl.empty[stage]), 3);
+                        if (++stage == G::STAGES) { stage = 0; phase ^= 1u; }
                     }
                     if (!ok) break;
-                    ptx::umma_commit(ptx::smem_u32(&ctl.tfull[acc]));         // accumulator complete
+                    // accumulator complete (in both CTAs of a pair)
+                    if (CG == 1) ptx::umma_commit(ptx::smem_u32(&ctl.tfull[acc]));
+                    else ptx::umma_commit_pair(ptx::smem_u32(&ctl.tfull[acc]), 3);
                     acc ^= 1u;
                     if (acc == 0) acc_phase ^= 1u;
                 }
             }
             if (!ok) {
                 // aborted: make sure no MMA is still in flight before TMEM is freed
-                ptx::umma_commit(ptx::smem_u32(&ctl.drain));
+                if (CG == 1) ptx::umma_commit(ptx::smem_u32(&ctl.drain));
+                else ptx::umma_commit_pair(ptx::smem_u32(&ctl.drain), 1);
                 wait_bounded(ptx::smem_u32(&ctl.drain), 0, abort, status, 20000000ull);
             }
         }
@@ -486,10 +546,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         typename Epi::State st;
-        for (int item = blockIdx.x; item < sched.n_items && ok; item += gridDim.x) {
+        for (int item = worker; item < sched.n_items && ok; item += n_workers) {
             int m_tile, group, n_begin, n_end;
             decode_item(sched, item, m_tile, group, n_begin, n_end);
-            Epi::begin_item(ep, st, m_tile, row_in_tile);
+            Epi::begin_item(ep, st, m_tile * CG + static_cast<int>(rank), row_in_tile);
             for (int n = n_begin; n < n_end; ++n) {
                 ok = wait_bounded(ptx::smem_u32(&ctl.tfull[acc]), acc_phase, abort, status);
                 ok = __all_sync(0xffffffffu, ok);
@@ -497,7 +557,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 ptx::tc_fence_after();
                 Epi::tile(ep, st, n, lane_base + acc * BN);
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(ptx::smem_u32(&ctl.tempty[acc]));
+                if (CG == 1) {
+                    ptx::mbar_arrive(ptx::smem_u32(&ctl.tempty[acc]));
+                } else {
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&ctl.tempty[acc]), 0));
+                }
                 acc ^= 1u;
                 if (acc == 0) acc_phase ^= 1u;
             }
@@ -505,11 +570,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     }
 
+    // Nothing of a pair may leave while its peer can still signal its barriers or read its
+    // shared memory, so the pair meets here before TMEM is returned.
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CG == 1) __syncthreads();
+    else ptx::cluster_sync_all();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc<TMEM_COLS>(tmem);
+        if (CG == 1) ptx::tmem_dealloc<TMEM_COLS>(tmem);
+        else ptx::tmem_dealloc_pair<TMEM_COLS>(tmem);
     }
 }
 

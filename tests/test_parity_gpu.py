@@ -145,9 +145,10 @@ def test_fused_reduced_configs_full_d_V_K(cfg, T):
 
 
 def test_fused_many_row_slabs_ragged_shapes_and_options():
-    batch = synth.make_batch(41, T=1000, d=200, V=5003 - 3, K=8)      # 8 slabs of 128 rows, ragged last slab
+    batch = synth.make_batch(41, T=1000, d=200, V=5003 - 3, K=8)      # one m-tile per slab, ragged last slab
     gpu, fwd = _fused_check(batch, slab_mib=1, g=0.1)
-    assert B.cat_loss_launch_count(gpu["obj"].shape, 2) == 1 + 8 * 5 + 1
+    n_launches = B.cat_loss_launch_count(gpu["obj"].shape, 2)         # scale + 5 per slab + finalize
+    assert (n_launches - 2) % 5 == 0 and (n_launches - 2) // 5 in (4, 8)   # slabs of 256 (CTA pairs) or 128 rows
     rng = np.random.default_rng(7)
     _fused_check(batch, slab_mib=2, conf_ext=rng.random(1000).astype(np.float32), use_valid=False)
     _, dH, dW = run_oracle(batch)
