@@ -32,6 +32,10 @@ Readings taken where the paper is silent (each also listed in the design notes):
     weight 0, no loss, no gradient, and factor 1 in the prefix product.
   * a label outside [0, V) on a valid row makes the row invalid.
 
+Beside the CAT objective: the fixed position decay gamma**k that the paper ablates CAT
+against (Table 3), the per-block acceptance-length estimate of Eq. 8, and the target-model
+confidences of Eq. 9 laid out as draft rows (Eq. 12's s_{n,k}).
+
 Pins (tests/test_oracle_pins.py): Eq. 5 degenerate case against
 torch.nn.functional.cross_entropy, K = 1, constant confidence = fixed decay
 gamma**k, W = 0 closed form, the Eq. 6/Eq. 8 acceptance-length identity, a hand
@@ -48,6 +52,11 @@ __all__ = [
     "softmax_stats",
     "cat_weights",
     "cat_weights_f32",
+    "fixed_decay_weights",
+    "fixed_decay_weights_f32",
+    "accept_len_estimate",
+    "target_confidence",
+    "window_confidence",
     "cat_forward",
     "cat_backward",
     "cat_forward_backward",
@@ -121,8 +130,78 @@ def cat_weights_f32(conf_f32: np.ndarray, eff_valid: np.ndarray, K: int) -> np.n
     return w.reshape(-1)
 
 
+def fixed_decay_weights(gamma: float, eff_valid: np.ndarray, K: int) -> np.ndarray:
+    """The fixed position decay the paper ablates CAT against (Section 4.3, Table 3):
+    the weight of draft position k is gamma**k whatever the confidences are; k counts
+    positions, so masked rows in between still advance the exponent.  Invalid rows get 0.
+    Sequential product (1*gamma)*gamma*..., float64."""
+    ok = np.asarray(eff_valid, dtype=bool).reshape(-1, K)
+    w = np.zeros(ok.shape, dtype=np.float64)
+    s = 1.0
+    for k in range(K):
+        w[:, k] = np.where(ok[:, k], s, 0.0)
+        s = s * float(gamma)
+    return w.reshape(-1)
+
+
+def fixed_decay_weights_f32(gamma, eff_valid: np.ndarray, K: int) -> np.ndarray:
+    """fixed_decay_weights in IEEE binary32: ((1*g)*g)*... with g = float32(gamma)."""
+    ok = np.asarray(eff_valid, dtype=bool).reshape(-1, K)
+    g = np.float32(gamma)
+    w = np.zeros(ok.shape, dtype=np.float32)
+    s = np.float32(1.0)
+    for k in range(K):
+        w[:, k] = np.where(ok[:, k], s, np.float32(0.0))
+        s = np.float32(s * g)
+    return w.reshape(-1)
+
+
+def accept_len_estimate(conf: np.ndarray, weight: np.ndarray, K: int) -> np.ndarray:
+    """Per-block estimate of the expected acceptance length, Eq. 8 with the estimates of
+    Eq. 9 and Eq. 10 in place of a_k and s_k:  sum_k s_k * c_k  (invalid rows have s_k = 0)."""
+    c = np.asarray(conf, dtype=np.float64).reshape(-1, K)
+    w = np.asarray(weight, dtype=np.float64).reshape(-1, K)
+    return (w * c).sum(axis=1)
+
+
+def target_confidence(Ht, Wt, labels, valid=None, row_chunk: int = 1024):
+    """Eq. 9: the probability the TARGET model gives the ground-truth token of every sequence
+    position, teacher-forced: c_i = softmax(Ht[i] . Wt^T)[y_i].  Ht [L, d_t] are the target's
+    final hidden states, Wt [V, d_t] its LM head.  Returns (conf[L], lse[L]); positions that
+    are masked or whose label is outside [0, V) get confidence 1."""
+    Hd, Wd, y = _as_f64(Ht), _as_f64(Wt), _as_i64(labels)
+    L = Hd.shape[0]
+    ok = effective_valid(y, valid, Wd.shape[0])
+    ysafe = np.where(ok, y, 0)
+    lse = np.empty(L)
+    zy = np.empty(L)
+    for r0 in range(0, L, row_chunk):
+        r1 = min(L, r0 + row_chunk)
+        z = Hd[r0:r1] @ Wd.T
+        _, _, lse[r0:r1] = softmax_stats(z)
+        zy[r0:r1] = z[np.arange(r1 - r0), ysafe[r0:r1]]
+    return np.where(ok, np.exp(zy - lse), 1.0), lse
+
+
+def window_confidence(conf_seq: np.ndarray, block_start, K: int) -> np.ndarray:
+    """Lay per-position target confidences out as draft rows (Eq. 12's s_{n,k}): the block that
+    drafts positions start..start+K-1 of the flattened sequence gets conf_ext[b*K + k] =
+    conf_seq[start_b + k]; positions outside [0, L) get 1 (those rows are invalid anyway).
+    Eq. 10 applied to these rows is the sliding-window product over the sequence."""
+    c = np.asarray(conf_seq, dtype=np.float64)
+    st = _as_i64(block_start)
+    L = c.shape[0]
+    out = np.ones((st.shape[0], K), dtype=np.float64)
+    for b in range(st.shape[0]):
+        for k in range(K):
+            i = int(st[b]) + k
+            if 0 <= i < L:
+                out[b, k] = c[i]
+    return out.reshape(-1)
+
+
 def cat_forward(H, W, labels, valid, K: int, conf_ext=None, row_chunk: int = 1024,
-                check_rows_sum_to_one: bool = True) -> dict:
+                check_rows_sum_to_one: bool = True, fixed_decay_gamma=None) -> dict:
     """Forward pass of the CAT objective (Eq. 9-11) over T = B*K rows.
 
     Returns a dict with float64 arrays lse[T], z_label[T], conf[T], weight[T],
@@ -151,7 +230,10 @@ def cat_forward(H, W, labels, valid, K: int, conf_ext=None, row_chunk: int = 102
         conf = np.where(ok, p_label, 1.0)           # Eq. 9 evaluated with this head
     else:
         conf = np.where(ok, _as_f64(conf_ext), 1.0)  # Eq. 9 from the target model, supplied
-    w = cat_weights(conf, ok, K)                    # Eq. 10
+    if fixed_decay_gamma is None:
+        w = cat_weights(conf, ok, K)                # Eq. 10
+    else:
+        w = fixed_decay_weights(fixed_decay_gamma, ok, K)   # the ablation baseline: gamma**k
     row_ce = np.where(ok, lse - zy, 0.0)            # -log P(y_r)
     n_valid = int(ok.sum())
     loss = float((w * row_ce).sum() / n_valid) if n_valid > 0 else 0.0   # Eq. 11, batch mean
@@ -186,8 +268,9 @@ def cat_backward(H, W, labels, K: int, fwd: dict, g: float = 1.0, row_chunk: int
 
 
 def cat_forward_backward(H, W, labels, valid, K: int, conf_ext=None, g: float = 1.0,
-                         row_chunk: int = 1024):
-    fwd = cat_forward(H, W, labels, valid, K, conf_ext=conf_ext, row_chunk=row_chunk)
+                         row_chunk: int = 1024, fixed_decay_gamma=None):
+    fwd = cat_forward(H, W, labels, valid, K, conf_ext=conf_ext, row_chunk=row_chunk,
+                      fixed_decay_gamma=fixed_decay_gamma)
     dH, dW = cat_backward(H, W, labels, K, fwd, g=g, row_chunk=row_chunk)
     return fwd, dH, dW
 

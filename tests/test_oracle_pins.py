@@ -85,6 +85,121 @@ def test_constant_confidence_is_fixed_decay():
         assert math.isclose(fwd["loss"], float((expect * ce).mean()), rel_tol=1e-13)
 
 
+# ---------------------------------------------------------------- fixed position decay (Table 3 baseline)
+def _read_decay_examples():
+    out = []
+    with open(os.path.join(GOLDEN, "fixed_decay_hand_examples.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, g, v, w = [p.strip() for p in line.split("|")]
+            out.append((int(k), float(g), np.array(v.split(), int), np.array(w.split(), float)))
+    return out
+
+
+@pytest.mark.parametrize("K,gamma,v,w", _read_decay_examples())
+def test_fixed_decay_hand_examples(K, gamma, v, w):
+    assert np.array_equal(O.fixed_decay_weights(gamma, v.astype(bool), K), w)
+    assert np.array_equal(O.fixed_decay_weights_f32(gamma, v.astype(bool), K), w.astype(np.float32))
+
+
+def test_fixed_decay_matches_closed_form_and_the_constant_confidence_case():
+    H, W, y, valid = _rand_problem(13, 5 * 8, 8, 32)
+    for gamma in (1.0, 0.8, 0.6):                       # the three rates of Table 3
+        fwd, dH, dW = O.cat_forward_backward(H, W, y, valid, 8, fixed_decay_gamma=gamma)
+        assert np.allclose(fwd["weight"].reshape(-1, 8), gamma ** np.arange(8), rtol=1e-14)
+        # with every row valid it is CAT with all confidences equal to gamma
+        ref, dH2, dW2 = O.cat_forward_backward(H, W, y, valid, 8, conf_ext=np.full(40, gamma))
+        assert math.isclose(fwd["loss"], ref["loss"], rel_tol=1e-13)
+        assert np.allclose(dH, dH2, rtol=1e-12, atol=1e-18) and np.allclose(dW, dW2, rtol=1e-12, atol=1e-18)
+    # gamma = 1 is the uniform loss of Eq. 5
+    one = O.cat_forward(H, W, y, valid, 8, fixed_decay_gamma=1.0)
+    loss_t, _, _ = _torch_ce(H, W, y, valid, 40)
+    assert math.isclose(one["loss"], loss_t, rel_tol=1e-12)
+    # the model's own confidences are still reported, and play no part in the weights
+    assert np.allclose(one["conf"], np.exp(one["z_label"] - one["lse"]), rtol=1e-14)
+
+
+def test_fixed_decay_counts_positions_not_valid_rows():
+    ok = np.array([1, 0, 0, 1, 1, 1, 0, 1], bool)
+    w = O.fixed_decay_weights(0.5, ok, 4).reshape(2, 4)
+    assert np.array_equal(w, [[1, 0, 0, 0.125], [1, 0.5, 0, 0.125]])
+    # CAT with constant confidence skips masked rows instead: the two differ exactly there
+    w_cat = O.cat_weights(np.full(8, 0.5), ok, 4).reshape(2, 4)
+    assert np.array_equal(w_cat, [[1, 0, 0, 0.5], [1, 0.5, 0, 0.25]])
+
+
+# ---------------------------------------------------------------- Eq. 8 estimate per block
+def test_accept_len_estimate_closed_forms():
+    K = 8
+    # constant confidence c: sum_k c^k * c = c (1 - c^K) / (1 - c)
+    for c in (0.9, 0.5, 0.1):
+        conf = np.full(3 * K, c)
+        w = O.cat_weights(conf, np.ones(3 * K, bool), K)
+        est = O.accept_len_estimate(conf, w, K)
+        assert np.allclose(est, c * (1 - c ** K) / (1 - c), rtol=1e-13)
+    # certain drafter: every token accepted, length K;  first token never accepted: length 0
+    ones = np.ones(K)
+    assert O.accept_len_estimate(ones, O.cat_weights(ones, ones.astype(bool), K), K)[0] == K
+    c0 = np.array([0.0] + [0.7] * (K - 1))
+    assert O.accept_len_estimate(c0, O.cat_weights(c0, np.ones(K, bool), K), K)[0] == 0.0
+    # Eq. 3 by brute force: E[L] = sum over acceptance patterns of (prefix length * probability)
+    rng = np.random.default_rng(5)
+    c = rng.random(4)
+    brute = 0.0
+    for bits in range(16):
+        acc = [(bits >> k) & 1 for k in range(4)]
+        prob = np.prod([c[k] if acc[k] else 1 - c[k] for k in range(4)])
+        length = 0
+        while length < 4 and acc[length]:
+            length += 1
+        brute += prob * length
+    est = O.accept_len_estimate(c, O.cat_weights(c, np.ones(4, bool), 4), 4)[0]
+    assert math.isclose(est, brute, rel_tol=1e-13)
+
+
+# ---------------------------------------------------------------- Eq. 9 with a target head, Eq. 12 layout
+def test_target_confidence_is_softmax_probability_of_the_label():
+    rng = np.random.default_rng(21)
+    L, dt, V = 19, 6, 11
+    Ht, Wt = rng.standard_normal((L, dt)), rng.standard_normal((V, dt))
+    y = rng.integers(0, V, L)
+    y[3] = -100
+    conf, lse = O.target_confidence(Ht, Wt, y)
+    p = torch.softmax(torch.tensor(Ht @ Wt.T), dim=1).numpy()
+    for i in range(L):
+        assert math.isclose(conf[i], 1.0 if i == 3 else p[i, y[i]], rel_tol=1e-13)
+    assert np.allclose(lse, torch.logsumexp(torch.tensor(Ht @ Wt.T), dim=1).numpy(), rtol=1e-14)
+    # Wt = 0: every token has probability 1/V
+    c0, l0 = O.target_confidence(Ht, np.zeros((V, dt)), y)
+    assert np.allclose(np.delete(c0, 3), 1.0 / V, rtol=1e-14) and np.allclose(l0, math.log(V), rtol=1e-14)
+
+
+def test_window_confidence_gives_the_sliding_product_of_eq12():
+    # a sequence of L positions with confidences c_i; the block that starts at position n holds
+    # c_n..c_{n+K-1}, so Eq. 10 on it gives s_{n,k} = prod_{j<k} c_{n+j}: a window sliding with n
+    rng = np.random.default_rng(22)
+    L, K = 12, 4
+    c = rng.random(L)
+    starts = np.arange(0, L)                 # one block per prefix position
+    ce = O.window_confidence(c, starts, K)
+    assert ce.shape == (L * K,)
+    ok = np.array([[n + k < L for k in range(K)] for n in starts]).reshape(-1)   # Eq. 12: n <= N - k
+    w = O.cat_weights(ce, ok, K).reshape(L, K)
+    for n in range(L):
+        for k in range(K):
+            if n + k < L:
+                assert ce[n * K + k] == c[n + k]
+                assert math.isclose(w[n, k], float(np.prod(c[n:n + k])), rel_tol=1e-14)
+            else:
+                assert ce[n * K + k] == 1.0 and w[n, k] == 0.0
+    # the same target position carries the same confidence in every block that contains it
+    assert ce[0 * K + 3] == ce[1 * K + 2] == ce[2 * K + 1] == ce[3 * K + 0] == c[3]
+    # a start before the sequence or past its end reads as 1
+    assert np.array_equal(O.window_confidence(c, np.array([-2, L - 1]), K), [1, 1, c[0], c[1], c[L - 1], 1, 1, 1])
+
+
 # ---------------------------------------------------------------- Eq. 5 / Eq. 11 degenerate cases
 def _torch_ce(H, W, y, valid, reduction_n):
     Ht = torch.tensor(H, dtype=torch.float64, requires_grad=True)
