@@ -62,6 +62,13 @@ typedef enum {
 
 typedef enum { CAT_BF16 = 0, CAT_F32 = 1 } cat_dtype;
 
+/* How the per-row weight is formed. */
+typedef enum {
+    CAT_WEIGHT_CONFIDENCE = 0,   /* Eq. 10: exclusive product of the confidences of the block's earlier rows */
+    CAT_WEIGHT_FIXED_DECAY = 1   /* decay_gamma^k for draft position k: the fixed position-wise decay the
+                                    paper compares CAT with (Section 4.3, Table 3, gamma_t = gamma^(t-1))   */
+} cat_weight_mode;
+
 /* Problem description, read on the host. */
 typedef struct {
     int64_t T;         /* rows = draft blocks * K                                   */
@@ -76,6 +83,11 @@ typedef struct {
                           Smaller caps mean more, smaller slabs.                          */
     int64_t ldH;       /* row pitch of H and dH in elements, >= d                     */
     int64_t ldW;       /* row pitch of W and dW in elements, >= d                     */
+    int32_t weight_mode;  /* cat_weight_mode; 0 = the CAT weights of Eq. 10                */
+    float   decay_gamma;  /* CAT_WEIGHT_FIXED_DECAY only: weight of position k is the binary32
+                             product ((1*gamma)*gamma)*... of k factors; k counts positions, so a
+                             masked row still moves the exponent on.  Must be finite and >= 0.
+                             conf[] still reports the head's (or conf_ext's) confidences.        */
 } cat_shape;
 
 /* Per-call statistics written by cat_loss_fwd (device memory, 32 bytes). */
@@ -90,7 +102,7 @@ typedef struct {
 
 /*
  * Bytes of scratch the given pass needs for this shape: pass 0 = cat_loss_fwd,
- * pass 1 = cat_loss_bwd, pass 2 = cat_loss_fwd_bwd.  Returns 0 if the shape is invalid.  The scratch holds the
+ * pass 1 = cat_loss_bwd, pass 2 = cat_loss_fwd_bwd, pass 3 = cat_conf_fwd.  Returns 0 if the shape is invalid.  The scratch holds the
  * per-(row, vocabulary split) softmax partials in the forward pass, and in the backward
  * pass one bounded slab of dz (bf16: rows x a slice of the vocabulary, at most about
  * 2 GiB) plus an fp32 dH accumulator when the vocabulary is processed in more than one
@@ -194,6 +206,49 @@ int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W,
                         const int64_t* labels, const uint8_t* valid, const float* conf_ext,
                         float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
                         void* cuda_stream);
+
+/*
+ * Per-block estimate of the expected acceptance length, Eq. 8 with the estimates of Eq. 9 and
+ * Eq. 10 in place of the acceptance rates:  accept_len[b] = sum_k weight[bK+k] * conf[bK+k].
+ * (cat_stats.est_accept_len is the mean of these.)  Only T and K of `shape` are used.
+ *   conf, weight  [T] fp32 as written by cat_loss_fwd / cat_loss_fwd_bwd       (device, in)
+ *   accept_len    [T / K] fp32                                                  (device, out)
+ * One kernel, no workspace.  Returns CAT_OK or a negative cat_status.
+ */
+int cat_accept_len(const cat_shape* shape, const float* conf, const float* weight, float* accept_len,
+                   void* cuda_stream);
+
+/*
+ * Confidence producer for the paper's own reading of Eq. 9: the probability that the TARGET
+ * model gives the ground-truth token at every position of the (flattened) training sequences,
+ *     conf_seq[i] = softmax(Ht[i, :] . Wt^T)[labels[i]],
+ * computed with the same vocabulary-chunked GEMM and online softmax as cat_loss_fwd, never
+ * storing the logits.  `shape` describes the target head: T = number of positions L, d = the
+ * target's hidden size, V, in_dtype, ldH/ldW pitches; K, dW_dtype and weight_mode are ignored.
+ *   Ht, Wt     [L, d], [V, d] target hidden states and target LM head            (device, in)
+ *   labels     [L] int64: the token that follows position i's prefix               (device, in)
+ *   valid      [L] uint8 or NULL                                                   (device, in)
+ *   conf_seq   [L] fp32 (1 for masked positions / labels outside [0, V))           (device, out)
+ *   lse_seq    [L] fp32 log-sum-exp of the target logits                           (device, out)
+ *   workspace  at least cat_loss_workspace_bytes(shape, 3) bytes, 256-byte aligned
+ * Returns CAT_OK or a negative cat_status; the workspace's first int32 holds the device status.
+ */
+int cat_conf_fwd(const cat_shape* shape, const void* Ht, const void* Wt, const int64_t* labels,
+                 const uint8_t* valid, float* conf_seq, float* lse_seq,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Lays per-position confidences out as draft rows, which turns Eq. 10 into the prefix-indexed
+ * weight s_{n,k} of Eq. 12 (a product over a window that slides with the prefix position n):
+ *     conf_ext[b*K + k] = conf_seq[block_start[b] + k]   if 0 <= block_start[b] + k < L, else 1.
+ * Pass the result as `conf_ext` to cat_loss_fwd / cat_loss_fwd_bwd.
+ *   conf_seq     [L] fp32                                                         (device, in)
+ *   block_start  [n_blocks] int64: index in conf_seq of the block's first drafted token (device, in)
+ *   conf_ext     [n_blocks * K] fp32                                              (device, out)
+ * One kernel, no workspace.  Returns CAT_OK or a negative cat_status.
+ */
+int cat_conf_window(const float* conf_seq, int64_t L, const int64_t* block_start, int64_t n_blocks,
+                    int32_t K, float* conf_ext, void* cuda_stream);
 
 /*
  * Number of kernels of this library that the given pass (0 = cat_loss_fwd, 1 = cat_loss_bwd,

@@ -14,12 +14,17 @@ class CatLoss:
     """Buffers and calls for one (T, d, V, K, dtype) problem on the current CUDA device."""
 
     def __init__(self, T: int, d: int, V: int, K: int, dtype: torch.dtype = torch.bfloat16,
-                 dW_dtype: torch.dtype = torch.float32, slab_mib: int = 0, device: str = "cuda"):
+                 dW_dtype: torch.dtype = torch.float32, slab_mib: int = 0, device: str = "cuda",
+                 fixed_decay_gamma: float | None = None):
         if not torch.cuda.is_available():
             raise RuntimeError("CatLoss needs a CUDA device; there is no CPU path")
         code = {torch.bfloat16: B.CAT_BF16, torch.float32: B.CAT_F32}
         self.dtype, self.dW_dtype = dtype, dW_dtype
-        self.shape = B.make_shape(T, d, V, K, code[dtype], code[dW_dtype], slab_mib=slab_mib)
+        if fixed_decay_gamma is None:
+            self.shape = B.make_shape(T, d, V, K, code[dtype], code[dW_dtype], slab_mib=slab_mib)
+        else:   # the fixed position decay the paper compares CAT with: weight gamma^k
+            self.shape = B.make_shape(T, d, V, K, code[dtype], code[dW_dtype], slab_mib=slab_mib,
+                                      weight_mode=B.CAT_WEIGHT_FIXED_DECAY, decay_gamma=float(fixed_decay_gamma))
         self.T, self.d, self.V, self.K = T, d, V, K
         dev = torch.device(device)
         nf, nb = B.cat_loss_workspace_bytes(self.shape, 0), B.cat_loss_workspace_bytes(self.shape, 1)
@@ -55,6 +60,13 @@ class CatLoss:
                            self.weight, self.stats, self.dH, self.dW, accumulate_dW, self._ws_fused)
         return self.loss, self.dH, self.dW
 
+    def accept_len(self) -> torch.Tensor:
+        """cat_accept_len: per-block estimate of the expected acceptance length (Eq. 8) from the
+        conf / weight of the last forward."""
+        out = torch.empty(self.T // self.K, dtype=torch.float32, device=self.loss.device)
+        B.cat_accept_len(self.shape, self.conf, self.weight, out)
+        return out
+
     def fused_status(self) -> int:
         return int(self._ws_fused[:4].view(torch.int32).item())
 
@@ -63,3 +75,35 @@ class CatLoss:
 
     def fwd_stats(self):
         return B.read_stats(self.stats)
+
+
+class TargetConfidence:
+    """Buffers and calls for cat_conf_fwd / cat_conf_window: target-model confidences of L
+    sequence positions (Eq. 9) and their layout as draft rows (Eq. 12)."""
+
+    def __init__(self, L: int, d: int, V: int, dtype: torch.dtype = torch.bfloat16, device: str = "cuda"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("TargetConfidence needs a CUDA device; there is no CPU path")
+        code = {torch.bfloat16: B.CAT_BF16, torch.float32: B.CAT_F32}
+        self.L = L
+        self.shape = B.make_shape(L, d, V, 1, code[dtype])
+        n = B.cat_loss_workspace_bytes(self.shape, 3)
+        if n == 0:
+            raise ValueError("invalid shape for cat_conf_fwd")
+        dev = torch.device(device)
+        self.ws = torch.empty(n, dtype=torch.uint8, device=dev)
+        self.conf_seq = torch.empty(L, dtype=torch.float32, device=dev)
+        self.lse_seq = torch.empty(L, dtype=torch.float32, device=dev)
+
+    def forward(self, Ht, Wt, labels, valid=None):
+        B.cat_conf_fwd(self.shape, Ht, Wt, labels, valid, self.conf_seq, self.lse_seq, self.ws)
+        return self.conf_seq
+
+    def window(self, block_start: torch.Tensor, K: int) -> torch.Tensor:
+        n_blocks = block_start.numel()
+        out = torch.empty(n_blocks * K, dtype=torch.float32, device=self.conf_seq.device)
+        B.cat_conf_window(self.conf_seq, self.L, block_start, n_blocks, K, out)
+        return out
+
+    def status(self) -> int:
+        return int(self.ws[:4].view(torch.int32).item())

@@ -14,13 +14,15 @@ import torch
 from . import build as _build
 
 CAT_BF16, CAT_F32 = 0, 1
+CAT_WEIGHT_CONFIDENCE, CAT_WEIGHT_FIXED_DECAY = 0, 1
 CAT_OK = 0
 
 
 class cat_shape(ctypes.Structure):
     _fields_ = [("T", ctypes.c_int64), ("d", ctypes.c_int64), ("V", ctypes.c_int64), ("K", ctypes.c_int32),
                 ("in_dtype", ctypes.c_int32), ("dW_dtype", ctypes.c_int32), ("slab_mib", ctypes.c_int32),
-                ("ldH", ctypes.c_int64), ("ldW", ctypes.c_int64)]
+                ("ldH", ctypes.c_int64), ("ldW", ctypes.c_int64), ("weight_mode", ctypes.c_int32),
+                ("decay_gamma", ctypes.c_float)]
 
 
 class cat_stats(ctypes.Structure):
@@ -58,6 +60,12 @@ def lib() -> ctypes.CDLL:
         L.cat_loss_fwd_bwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 13 + [ctypes.c_int, vp, sz, vp]
         L.cat_loss_bwd.restype = ctypes.c_int
         L.cat_loss_bwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 9 + [ctypes.c_int, vp, sz, vp]
+        L.cat_accept_len.restype = ctypes.c_int
+        L.cat_accept_len.argtypes = [ctypes.POINTER(cat_shape), vp, vp, vp, vp]
+        L.cat_conf_fwd.restype = ctypes.c_int
+        L.cat_conf_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 6 + [vp, sz, vp]
+        L.cat_conf_window.restype = ctypes.c_int
+        L.cat_conf_window.argtypes = [vp, ctypes.c_int64, vp, ctypes.c_int64, ctypes.c_int32, vp, vp]
         _lib = L
     return _lib
 
@@ -66,8 +74,10 @@ def cat_status_string(code: int) -> str:
     return lib().cat_status_string(int(code)).decode()
 
 
-def make_shape(T, d, V, K, in_dtype, dW_dtype=CAT_F32, ldH=None, ldW=None, slab_mib=0) -> cat_shape:
-    return cat_shape(T, d, V, K, in_dtype, dW_dtype, slab_mib, d if ldH is None else ldH, d if ldW is None else ldW)
+def make_shape(T, d, V, K, in_dtype, dW_dtype=CAT_F32, ldH=None, ldW=None, slab_mib=0,
+               weight_mode=CAT_WEIGHT_CONFIDENCE, decay_gamma=0.0) -> cat_shape:
+    return cat_shape(T, d, V, K, in_dtype, dW_dtype, slab_mib, d if ldH is None else ldH, d if ldW is None else ldW,
+                     weight_mode, decay_gamma)
 
 
 def cat_loss_workspace_bytes(shape: cat_shape, which: int) -> int:
@@ -126,6 +136,26 @@ def cat_loss_fwd_bwd(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse,
                                 workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_loss_fwd_bwd")
+
+
+def cat_accept_len(shape, conf, weight, accept_len) -> None:
+    rc = lib().cat_accept_len(ctypes.byref(shape), _ptr(conf), _ptr(weight), _ptr(accept_len), _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_accept_len")
+
+
+def cat_conf_fwd(shape, Ht, Wt, labels, valid, conf_seq, lse_seq, workspace) -> None:
+    rc = lib().cat_conf_fwd(ctypes.byref(shape), _ptr(Ht), _ptr(Wt), _ptr(labels), _ptr(valid), _ptr(conf_seq),
+                            _ptr(lse_seq), _ptr(workspace),
+                            workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_conf_fwd")
+
+
+def cat_conf_window(conf_seq, L, block_start, n_blocks, K, conf_ext) -> None:
+    rc = lib().cat_conf_window(_ptr(conf_seq), int(L), _ptr(block_start), int(n_blocks), int(K), _ptr(conf_ext), _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_conf_window")
 
 
 def read_stats(stats_tensor: torch.Tensor) -> cat_stats:

@@ -10,6 +10,8 @@
 
 #include <stdlib.h>
 
+#include <math.h>
+
 #include <mutex>
 
 #include "rowops.cuh"
@@ -54,6 +56,8 @@ int check_shape(const cat_shape* s) {
     if (s->in_dtype != CAT_BF16 && s->in_dtype != CAT_F32) return CAT_ERR_DTYPE;
     if (s->dW_dtype != CAT_BF16 && s->dW_dtype != CAT_F32) return CAT_ERR_DTYPE;
     if (s->in_dtype == CAT_F32 && s->dW_dtype != CAT_F32) return CAT_ERR_DTYPE;
+    if (s->weight_mode != CAT_WEIGHT_CONFIDENCE && s->weight_mode != CAT_WEIGHT_FIXED_DECAY) return CAT_ERR_SHAPE;
+    if (s->weight_mode == CAT_WEIGHT_FIXED_DECAY && !(s->decay_gamma >= 0.f && s->decay_gamma <= 3.0e38f)) return CAT_ERR_SHAPE;
     if (s->in_dtype == CAT_BF16 && (s->d % 8 != 0 || s->ldH % 8 != 0 || s->ldW % 8 != 0)) return CAT_ERR_ALIGN;
     return CAT_OK;
 }
@@ -312,6 +316,16 @@ tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int b
     return s;
 }
 
+// cat_conf_fwd treats every sequence position as a draft block of its own (K = 1, Eq. 10 weights).
+cat_shape per_position_shape(const cat_shape* s) {
+    cat_shape one = *s;
+    one.K = 1;
+    one.dW_dtype = CAT_F32;
+    one.weight_mode = CAT_WEIGHT_CONFIDENCE;
+    one.decay_gamma = 0.f;
+    return one;
+}
+
 }  // namespace
 
 // =================================================================================== exports
@@ -342,6 +356,10 @@ size_t cat_loss_workspace_bytes(const cat_shape* shape, int pass) {
         const size_t a = plan_fwd(shape).total, b = plan_bwd(shape).total;
         return a > b ? a : b;
     }
+    if (pass == 3) {
+        const cat_shape one = per_position_shape(shape);
+        return align256(plan_fwd(&one).total) + align256(sizeof(float) * (static_cast<size_t>(one.T) + 64));
+    }
     return 0;
 }
 
@@ -349,6 +367,7 @@ int cat_loss_launch_count(const cat_shape* shape, int pass) {
     if (check_shape(shape) != CAT_OK) return 0;
     if (pass == 0) return 1 + (plan_fwd(shape).warp_scan ? 1 : 2) + 1;
     if (pass == 1) return 1 + 3 * plan_bwd(shape).n_slabs;
+    if (pass == 3) return 3;
     if (pass == 2) {
         if (shape->in_dtype != CAT_BF16)
             return cat_loss_launch_count(shape, 0) + cat_loss_launch_count(shape, 1);
@@ -419,6 +438,7 @@ int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int
     rp.labels = reinterpret_cast<const long long*>(labels); rp.valid = valid; rp.conf_ext = conf_ext;
     rp.lse = lse; rp.conf = conf; rp.weight = weight; rp.row_ce = row_ce; rp.partials = partials;
     rp.T = T; rp.V = V; rp.K = shape->K; rp.S = plan.S; rp.part_stride = T;
+    rp.fixed_decay = shape->weight_mode == CAT_WEIGHT_FIXED_DECAY; rp.gamma = shape->decay_gamma;
     if (plan.warp_scan) {
         rows::row_kernel<true><<<plan.n_row_ctas, rows::ROW_THREADS, 0, st>>>(rp);
     } else {
@@ -633,6 +653,7 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const
             rp.lse = lse + r0; rp.conf = conf + r0; rp.weight = weight + r0; rp.row_ce = row_ce + r0;
             rp.partials = partials + cta0; rp.part_stride = T;
             rp.T = static_cast<int>(rws); rp.V = V; rp.K = shape->K; rp.S = S;
+            rp.fixed_decay = shape->weight_mode == CAT_WEIGHT_FIXED_DECAY; rp.gamma = shape->decay_gamma;
             if (plan.warp_scan) {
                 n_ctas = static_cast<int>(cdiv(rws, rows::ROW_THREADS));
                 rows::row_kernel<true><<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
@@ -683,6 +704,45 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const
     }
     rows::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(partials, cta0, T / shape->K, loss,
                                                          reinterpret_cast<rows::StatsOut*>(stats), status);
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+}
+
+int cat_accept_len(const cat_shape* shape, const float* conf, const float* weight, float* accept_len, void* cuda_stream) {
+    if (!shape || !conf || !weight || !accept_len) return CAT_ERR_NULL;
+    if (shape->T <= 0 || shape->K < 1 || shape->T % shape->K != 0 || shape->T >= (1ll << 31)) return CAT_ERR_SHAPE;
+    if (misaligned(conf, 4) || misaligned(weight, 4) || misaligned(accept_len, 4)) return CAT_ERR_ALIGN;
+    const int n_blocks = static_cast<int>(shape->T / shape->K);
+    rows::accept_len_kernel<<<static_cast<unsigned>(cdiv(n_blocks, rows::ROW_THREADS)), rows::ROW_THREADS, 0,
+                              static_cast<cudaStream_t>(cuda_stream)>>>(conf, weight, accept_len, n_blocks, shape->K);
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+}
+
+int cat_conf_fwd(const cat_shape* shape, const void* Ht, const void* Wt, const int64_t* labels, const uint8_t* valid,
+                 float* conf_seq, float* lse_seq, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!shape || !Ht || !Wt || !labels || !conf_seq || !lse_seq) return CAT_ERR_NULL;
+    const cat_shape one = per_position_shape(shape);
+    const int sc = check_shape(&one);
+    if (sc != CAT_OK) return sc;
+    const size_t fwd_bytes = align256(plan_fwd(&one).total);
+    const size_t need = fwd_bytes + align256(sizeof(float) * (static_cast<size_t>(one.T) + 64));
+    if (!workspace || misaligned(workspace, 256) || workspace_bytes < need) return CAT_ERR_WORKSPACE;
+    // with K = 1 every weight is 1 and the loss is the target's own mean cross-entropy: both land in scratch
+    float* tail = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + fwd_bytes);
+    float* loss_tmp = tail;
+    float* weight_tmp = tail + 64;
+    return cat_loss_fwd(&one, Ht, Wt, labels, valid, nullptr, loss_tmp, lse_seq, conf_seq, weight_tmp, nullptr, workspace,
+                        fwd_bytes, cuda_stream);
+}
+
+int cat_conf_window(const float* conf_seq, int64_t L, const int64_t* block_start, int64_t n_blocks, int32_t K,
+                    float* conf_ext, void* cuda_stream) {
+    if (!conf_seq || !block_start || !conf_ext) return CAT_ERR_NULL;
+    if (L <= 0 || n_blocks <= 0 || K < 1 || n_blocks * K >= (1ll << 31)) return CAT_ERR_SHAPE;
+    if (misaligned(conf_seq, 4) || misaligned(block_start, 8) || misaligned(conf_ext, 4)) return CAT_ERR_ALIGN;
+    const long long n_rows = n_blocks * K;
+    rows::conf_window_kernel<<<static_cast<unsigned>(cdiv(n_rows, rows::ROW_THREADS)), rows::ROW_THREADS, 0,
+                               static_cast<cudaStream_t>(cuda_stream)>>>(conf_seq, L, reinterpret_cast<const long long*>(block_start),
+                                                                         n_rows, K, conf_ext);
     return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
 }
 

@@ -37,6 +37,8 @@ struct RowParams {
     CtaPartial* partials;      // [gridDim.x]
     long long part_stride;     // row pitch of the partial arrays (>= T)
     int T, V, K, S;
+    int fixed_decay;           // 0: Eq. 10 (product of confidences); 1: gamma^k by position
+    float gamma;
 };
 
 __device__ __forceinline__ void block_reduce_store(double loss, double sw, double swc, long long nv, long long nb,
@@ -95,13 +97,15 @@ __global__ void __launch_bounds__(ROW_THREADS) row_kernel(const RowParams p) {
         p.conf[r] = c;
     }
     if (SCAN) {
-        // Eq. 10: weight_k = ((1 * c_0) * c_1) ... * c_{k-1}; invalid rows carry the factor 1
+        // Eq. 10: weight_k = ((1 * c_0) * c_1) ... * c_{k-1}; invalid rows carry the factor 1.
+        // Fixed decay: every position carries the factor gamma instead.
         const int lane = threadIdx.x & 31;
         const int k = lane & (p.K - 1);
         const int base = lane - k;
+        const float factor = p.fixed_decay ? p.gamma : c;
         float run = 1.f;
         for (int j = 0; j + 1 < p.K; ++j) {
-            const float cj = __shfl_sync(0xffffffffu, c, base + j);
+            const float cj = __shfl_sync(0xffffffffu, factor, base + j);
             if (k > j) run = run * cj;
         }
         const float w = ok ? run : 0.f;
@@ -130,7 +134,8 @@ __global__ void __launch_bounds__(ROW_THREADS) block_scan_kernel(const RowParams
             const float c = p.conf[r];
             const float w = ok ? run : 0.f;
             p.weight[r] = w;
-            if (ok) run = run * c;
+            if (p.fixed_decay) run = run * p.gamma;
+            else if (ok) run = run * c;
             loss += static_cast<double>(w) * static_cast<double>(p.row_ce[r]);
             sw += w;
             swc += static_cast<double>(w) * c;
@@ -179,6 +184,31 @@ __global__ void __launch_bounds__(ROW_THREADS) finalize_kernel(const CtaPartial*
             stats->reserved = 0;
         }
     }
+}
+
+// Eq. 8 estimate per draft block: accept_len[b] = sum_k weight * conf, added in position order.
+__global__ void __launch_bounds__(ROW_THREADS) accept_len_kernel(const float* conf, const float* weight, float* out,
+                                                                 int n_blocks, int K) {
+    const int b = blockIdx.x * ROW_THREADS + threadIdx.x;
+    if (b >= n_blocks) return;
+    float acc = 0.f;
+    for (int k = 0; k < K; ++k) {
+        const size_t r = static_cast<size_t>(b) * K + k;
+        acc = fmaf(weight[r], conf[r], acc);
+    }
+    out[b] = acc;
+}
+
+// Eq. 12 layout: draft row (block b, position k) takes the confidence of sequence position
+// block_start[b] + k; positions outside the sequence read as 1.
+__global__ void __launch_bounds__(ROW_THREADS) conf_window_kernel(const float* conf_seq, long long L,
+                                                                  const long long* block_start, long long n_rows, int K,
+                                                                  float* conf_ext) {
+    const long long r = static_cast<long long>(blockIdx.x) * ROW_THREADS + threadIdx.x;
+    if (r >= n_rows) return;
+    const long long b = r / K;
+    const long long i = block_start[b] + (r - b * K);
+    conf_ext[r] = (i >= 0 && i < L) ? conf_seq[i] : 1.f;
 }
 
 // Backward set-up, single CTA: N = number of valid rows, scale = g / N (0 when N = 0).

@@ -18,7 +18,7 @@ from dataclasses import dataclass
 import numpy as np
 import torch
 
-__all__ = ["CONFIGS", "Batch", "make_batch", "zipf_labels"]
+__all__ = ["CONFIGS", "Batch", "make_batch", "zipf_labels", "TargetSide", "make_target_side"]
 
 
 @dataclass(frozen=True)
@@ -126,3 +126,42 @@ def make_batch(cfg: int, T: int | None = None, d: int | None = None, V: int | No
     if spec.invalid > 0:
         labels = torch.where(valid.bool(), labels, torch.full_like(labels, -100))
     return Batch(spec, T, K, d, V, H.contiguous(), W.contiguous(), labels.contiguous(), valid, biased)
+
+
+@dataclass
+class TargetSide:
+    """Inputs of the target-model side for a batch: one flattened training sequence of L
+    positions whose drafted continuations are the batch's blocks."""
+    L: int
+    d_t: int
+    Ht: torch.Tensor            # [L, d_t] target final hidden states
+    Wt: torch.Tensor            # [V, d_t] target LM head
+    seq_labels: torch.Tensor    # [L] int64: token that follows each position's prefix
+    block_start: torch.Tensor   # [T / K] int64: sequence index of each block's first drafted token
+
+
+def make_target_side(batch: Batch, d_t: int = 0, seed_offset: int = 7919) -> TargetSide:
+    """Target-side stand-ins for `batch`: one block per prefix position n = 0..B-1 of a sequence
+    of L = B + K - 1 positions, block n drafting positions n..n+K-1 (Eq. 12's (n, k) grid).  The
+    labels of the draft rows are NOT changed; seq_labels[n + k] is set to the label of row
+    (n, 0) for k = 0 and drawn for the tail, so they are only consistent along k = 0 -- enough
+    for a synthetic head, whose rows are independent draws anyway."""
+    spec = batch.spec
+    d_t = d_t or batch.d
+    nb = batch.T // batch.K
+    L = nb + batch.K - 1
+    gen = torch.Generator(device="cpu").manual_seed(spec.seed + seed_offset)
+    Ht = torch.randn(L, d_t, generator=gen, dtype=torch.float32)
+    Wt = torch.randn(batch.V, d_t, generator=gen, dtype=torch.float32) * 0.02
+    tail = torch.randint(0, batch.V, (batch.K - 1,), generator=gen, dtype=torch.int64)
+    first = batch.labels.reshape(nb, batch.K)[:, 0].clamp(min=0)
+    seq_labels = torch.cat([first, tail]).contiguous()
+    dt = batch.torch_dtype
+    Wt = Wt.to(dt)
+    # make the target fairly sure of about half of the positions, so window products are not all ~V^-k
+    sure = torch.rand(L, generator=gen) < 0.5
+    amount = 4.0 + 10.0 * torch.rand(L, generator=gen)
+    rows = torch.nonzero(sure).squeeze(1)
+    Wy = Wt[seq_labels[rows]].double()
+    Ht[rows] += (Wy * (amount[rows].double() / (Wy * Wy).sum(dim=1)).unsqueeze(1)).float()
+    return TargetSide(L, d_t, Ht.to(dt).contiguous(), Wt.contiguous(), seq_labels, torch.arange(nb, dtype=torch.int64))

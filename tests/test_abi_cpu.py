@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_header():
-    assert ctypes.sizeof(B.cat_shape) == 56
+    assert ctypes.sizeof(B.cat_shape) == 64
     assert ctypes.sizeof(B.cat_stats) == 32
 
 
@@ -54,7 +54,9 @@ def test_workspace_sizes():
     fused = B.cat_loss_workspace_bytes(s, 2)
     assert 0 < fused < 0.62 * logits_bytes        # one slab of logits, at least two slabs per batch
     assert B.cat_loss_workspace_bytes(big, 2) < 0.1 * (131072 * 128256 * 2)
-    assert B.cat_loss_workspace_bytes(s, 3) == 0
+    conf_ws = B.cat_loss_workspace_bytes(s, 3)       # cat_conf_fwd: forward scratch + O(T)
+    assert fwd <= conf_ws < 2 * fwd + (1 << 20) and B.cat_loss_workspace_bytes(s, 4) == 0
+    assert B.cat_loss_launch_count(s, 3) == 3
     assert B.cat_loss_launch_count(s, 0) == 3 and B.cat_loss_launch_count(s, 1) == 7
     assert B.cat_loss_launch_count(s, 2) == 1 + 2 * 5 + 1
 
