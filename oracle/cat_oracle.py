@@ -62,6 +62,8 @@ __all__ = [
     "cat_forward_backward",
     "cat_dH_rows",
     "cat_dW_rows",
+    "kd_target_rows",
+    "cat_kd_forward_backward",
 ]
 
 
@@ -301,3 +303,90 @@ def cat_dW_rows(H, W, labels, fwd: dict, vocab_rows: np.ndarray, g: float = 1.0)
     p -= (y[:, None] == v[None, :]) & ok[:, None]
     coef = np.where(ok, g * fwd["weight"] / N, 0.0)
     return (p * coef[:, None]).T @ Hd
+
+
+# ------------------------------------------------------------------------------------------
+# Section 3.3, Eq. 12: the full PARD-2 training loss, cross-entropy plus distillation from
+# the target model, both under the same prefix-indexed weight s_{n,k}.
+#
+# Readings (the paper names the distillation loss without writing it out):
+#   * L^KD of a row is the forward KL divergence from the target's next-token distribution
+#     p^t to the draft's q, both plain softmaxes (temperature 1) over the shared vocabulary:
+#         L^KD = sum_v p^t_v (log p^t_v - log q_v).
+#     Its gradient w.r.t. the draft logits is q - p^t; the target side receives no gradient.
+#   * The target distribution of draft row (n, k) is the target's teacher-forced distribution at
+#     sequence position n + k: it depends on the absolute position only, so one target row
+#     serves every draft row that predicts that position.  Draft row (b, k) uses target row
+#     block_start[b] + k of Ht; a row whose target position falls outside [0, L) is invalid.
+#   * Batch normaliser as for Eq. 11: divide by N = number of valid rows.
+#   * The weights may come from the target's confidence in the label (Eq. 9 as printed:
+#     c = p^t[y]), from the draft's own (the default of the plain CAT entry points), or from
+#     the caller (conf_ext).  They are constants under differentiation either way.
+# ------------------------------------------------------------------------------------------
+def kd_target_rows(block_start, K: int, T: int) -> np.ndarray:
+    """Target row of every draft row: t[b*K + k] = block_start[b] + k."""
+    st = _as_i64(block_start)
+    if st.shape[0] * K != T:
+        raise ValueError("block_start must have T / K entries")
+    return (st[:, None] + np.arange(K)[None, :]).reshape(-1)
+
+
+def cat_kd_forward_backward(H, W, labels, valid, K: int, Ht, Wt, block_start, beta: float,
+                            conf_source: str = "target", conf_ext=None, g: float = 1.0,
+                            fixed_decay_gamma=None, want_grads: bool = True):
+    """loss = (1/N) sum_r s_r (beta * CE_r + KD_r)  (Eq. 12 summed over k and n), its parts, and
+    the gradients of g * loss w.r.t. H and W with s held constant.
+
+    Returns (fwd dict, dH, dW).  fwd has loss, loss_ce, loss_kd (each already divided by N, so
+    loss = beta*loss_ce + loss_kd), lse, lse_t (per draft row), conf, weight, row_ce, row_kd,
+    eff_valid, n_valid, target_row.
+    """
+    Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
+    Htd, Wtd = _as_f64(Ht), _as_f64(Wt)
+    T, d = Hd.shape
+    V = Wd.shape[0]
+    L = Htd.shape[0]
+    if Wtd.shape[0] != V or Wtd.shape[1] != Htd.shape[1] or T % K != 0:
+        raise ValueError("bad shapes")
+    t_row = kd_target_rows(block_start, K, T)
+    ok = effective_valid(y, valid, V) & (t_row >= 0) & (t_row < L)
+    ysafe = np.where(ok, y, 0)
+    tsafe = np.where(ok, t_row, 0)
+
+    z = Hd @ Wd.T                                    # draft logits, all rows (small cases only)
+    zt = Htd[tsafe] @ Wtd.T                          # target logits of each draft row's position
+    _, _, lse = softmax_stats(z)
+    _, _, lse_t = softmax_stats(zt)
+    logq = z - lse[:, None]
+    logp = zt - lse_t[:, None]
+    p_t = np.exp(logp)
+    q = np.exp(logq)
+    rows = np.arange(T)
+    row_ce = np.where(ok, -logq[rows, ysafe], 0.0)                       # L^CE
+    row_kd = np.where(ok, (p_t * (logp - logq)).sum(axis=1), 0.0)        # L^KD = KL(p^t || q)
+    if conf_ext is not None:
+        conf = np.where(ok, _as_f64(conf_ext), 1.0)
+    elif conf_source == "target":
+        conf = np.where(ok, p_t[rows, ysafe], 1.0)                       # Eq. 9 as printed
+    elif conf_source == "draft":
+        conf = np.where(ok, q[rows, ysafe], 1.0)
+    else:
+        raise ValueError("conf_source must be 'target' or 'draft'")
+    w = cat_weights(conf, ok, K) if fixed_decay_gamma is None else fixed_decay_weights(fixed_decay_gamma, ok, K)
+    N = int(ok.sum())
+    loss_ce = float((w * row_ce).sum() / N) if N else 0.0
+    loss_kd = float((w * row_kd).sum() / N) if N else 0.0
+    fwd = dict(loss=beta * loss_ce + loss_kd, loss_ce=loss_ce, loss_kd=loss_kd, lse=lse, lse_t=lse_t, conf=conf,
+               weight=w, row_ce=row_ce, row_kd=row_kd, eff_valid=ok, n_valid=N, target_row=t_row)
+    if not want_grads:
+        return fwd, None, None
+    dH = np.zeros((T, d))
+    dW = np.zeros((V, d))
+    if N:
+        onehot = np.zeros((T, V))
+        onehot[rows, ysafe] = 1.0
+        coef = np.where(ok, g * w / N, 0.0)
+        dz = coef[:, None] * (beta * (q - onehot) + (q - p_t))
+        dH = dz @ Wd
+        dW = dz.T @ Hd
+    return fwd, dH, dW

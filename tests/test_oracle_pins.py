@@ -395,3 +395,109 @@ def test_weights_f32_is_sequential_binary32_with_denormals():
     c = np.full(16, np.float32(2.0 ** -10), np.float32)
     w = O.cat_weights_f32(c, np.ones(16, bool), 16)
     assert w[14] == np.float32(2.0 ** -140) and w[14] != 0 and w[15] == 0
+
+
+# ---------------------------------------------------------------- Eq. 12: CE + KD under the CAT weight
+def _kd_problem(seed, B=5, K=4, d=8, dt=6, V=32, masked=False):
+    rng = np.random.default_rng(seed)
+    T, L = B * K, B + K - 1
+    H, W = rng.standard_normal((T, d)), rng.standard_normal((V, d)) * 0.3
+    Ht, Wt = rng.standard_normal((L, dt)), rng.standard_normal((V, dt)) * 0.5
+    y = rng.integers(0, V, T)
+    valid = np.ones(T, np.uint8)
+    if masked:
+        valid[rng.random(T) < 0.25] = 0
+    return H, W, y, valid, Ht, Wt, np.arange(B)
+
+
+def test_eq12_against_library_kl_and_cross_entropy_with_unit_weights():
+    H, W, y, valid, Ht, Wt, st = _kd_problem(31, masked=True)
+    K, beta = 4, 0.1
+    fwd, dH, dW = O.cat_kd_forward_backward(H, W, y, valid, K, Ht, Wt, st, beta, conf_ext=np.ones(len(y)))
+    t_row = O.kd_target_rows(st, K, len(y))
+    ok = valid.astype(bool)
+    Hg = torch.tensor(H, requires_grad=True)
+    Wg = torch.tensor(W, requires_grad=True)
+    logq = torch.log_softmax(Hg @ Wg.T, dim=1)
+    p_t = torch.softmax(torch.tensor(Ht[t_row] @ Wt.T), dim=1)
+    kd = torch.nn.functional.kl_div(logq, p_t, reduction="none").sum(dim=1)      # KL(p_t || q) per row
+    ce = torch.nn.functional.nll_loss(logq, torch.tensor(y), reduction="none")
+    m = torch.tensor(ok)
+    loss = ((beta * ce + kd) * m).sum() / m.sum()
+    loss.backward()
+    assert math.isclose(fwd["loss"], loss.item(), rel_tol=1e-12)
+    assert math.isclose(fwd["loss"], beta * fwd["loss_ce"] + fwd["loss_kd"], rel_tol=1e-14)
+    assert np.allclose(dH, Hg.grad.numpy(), rtol=1e-10, atol=1e-15)
+    assert np.allclose(dW, Wg.grad.numpy(), rtol=1e-10, atol=1e-15)
+    assert np.all(fwd["row_kd"] >= -1e-15)
+
+
+def test_eq12_special_targets():
+    H, W, y, valid, Ht, Wt, st = _kd_problem(32)
+    K, beta, T = 4, 0.1, len(y)
+    cat, dH_c, dW_c = O.cat_forward_backward(H, W, y, valid, K, conf_ext=np.full(T, 0.5))
+    # (a) a target that puts all its mass on the label: KL(onehot || q) = -log q_y = CE, so the loss is (1 + beta) CAT
+    t_row = O.kd_target_rows(st, K, T)
+    #     one target row serves several draft rows, so give every draft row its own position: block_start = b * K
+    Ht_a = np.zeros((T, 32)); Wt_a = 60.0 * np.eye(32)
+    Ht_a[np.arange(T), y] = 1.0
+    fa, dH_a, dW_a = O.cat_kd_forward_backward(H, W, y, valid, K, Ht_a, Wt_a, np.arange(T // K) * K, beta, conf_ext=np.full(T, 0.5))
+    assert math.isclose(fa["loss_kd"], cat["loss"], rel_tol=1e-12) and math.isclose(fa["loss"], (1 + beta) * cat["loss"], rel_tol=1e-12)
+    assert np.allclose(dH_a, (1 + beta) * dH_c, rtol=1e-10, atol=1e-16) and np.allclose(dW_a, (1 + beta) * dW_c, rtol=1e-10, atol=1e-16)
+    #     and with the target as confidence source (Eq. 9) a certain target gives unit weights
+    fa2, _, _ = O.cat_kd_forward_backward(H, W, y, valid, K, Ht_a, Wt_a, np.arange(T // K) * K, beta, want_grads=False)
+    assert np.allclose(fa2["weight"], 1.0, rtol=0, atol=1e-12)
+    # (b) a target equal to the draft: KD = 0 with zero gradient, leaving beta * CAT
+    fb, dH_b, dW_b = O.cat_kd_forward_backward(H, W, y, valid, K, H, W, np.arange(T // K) * K, beta, conf_ext=np.full(T, 0.5))
+    assert abs(fb["loss_kd"]) <= 1e-15 and math.isclose(fb["loss"], beta * cat["loss"], rel_tol=1e-12)
+    assert np.allclose(dH_b, beta * dH_c, rtol=1e-10, atol=1e-16) and np.allclose(dW_b, beta * dW_c, rtol=1e-10, atol=1e-16)
+    # (c) uniform target against a uniform draft (W = 0): KD = 0; against a non-uniform draft: KD = mean(-log q) - log V
+    fc, _, _ = O.cat_kd_forward_backward(H, np.zeros_like(W), y, valid, K, Ht, np.zeros_like(Wt), st, beta, conf_ext=np.ones(T), want_grads=False)
+    assert abs(fc["loss_kd"]) <= 1e-15
+    fd, _, _ = O.cat_kd_forward_backward(H, W, y, valid, K, Ht, np.zeros_like(Wt), st, beta, conf_ext=np.ones(T), want_grads=False)
+    z = H @ W.T
+    logq = z - np.log(np.exp(z).sum(axis=1, keepdims=True))
+    assert math.isclose(fd["loss_kd"], float((-logq.mean(axis=1) - math.log(32)).mean()), rel_tol=1e-12)
+
+
+def test_eq12_target_rows_are_shared_along_n_plus_k_and_weights_follow_eq9():
+    H, W, y, valid, Ht, Wt, st = _kd_problem(33, B=6, K=4)
+    K, T, L = 4, len(y), Ht.shape[0]
+    fwd, _, _ = O.cat_kd_forward_backward(H, W, y, valid, K, Ht, Wt, st, 0.1, want_grads=False)
+    t_row = fwd["target_row"].reshape(-1, K)
+    assert t_row[1, 2] == t_row[2, 1] == t_row[3, 0] == 3                        # (n, k) -> n + k
+    assert np.array_equal(fwd["lse_t"].reshape(-1, K)[1, 2], fwd["lse_t"].reshape(-1, K)[3, 0])
+    # Eq. 9 as printed: the confidence is the target's probability of the row's label
+    zt = Ht @ Wt.T
+    p_t = np.exp(zt - np.log(np.exp(zt).sum(axis=1, keepdims=True)))
+    expect_c = p_t[fwd["target_row"], y]
+    assert np.allclose(fwd["conf"], expect_c, rtol=1e-13)
+    assert np.array_equal(fwd["weight"], O.cat_weights(fwd["conf"], np.ones(T, bool), K))
+    # a block whose positions run past the end of the sequence: those rows are invalid
+    f2, dH2, _ = O.cat_kd_forward_backward(H, W, y, valid, K, Ht, Wt, st + 2, 0.1)
+    bad = (O.kd_target_rows(st + 2, K, T) >= L)
+    assert bad.any() and not f2["eff_valid"][bad].any() and f2["eff_valid"][~bad].all()
+    assert not dH2[bad].any() and f2["n_valid"] == int((~bad).sum())
+
+
+def test_eq12_gradients_match_finite_differences_with_frozen_weights():
+    H, W, y, valid, Ht, Wt, st = _kd_problem(34, B=3, K=4, masked=True)
+    K, beta, g = 4, 0.1, 0.7
+    fwd, dH, dW = O.cat_kd_forward_backward(H, W, y, valid, K, Ht, Wt, st, beta, g=g)
+    w, N = fwd["weight"], fwd["n_valid"]
+
+    def frozen(Hx, Wx):
+        f, _, _ = O.cat_kd_forward_backward(Hx, Wx, y, valid, K, Ht, Wt, st, beta, conf_ext=np.ones(len(y)), want_grads=False)
+        return g * float((w * (beta * f["row_ce"] + f["row_kd"])).sum() / N)
+
+    eps = 1e-6
+    rng = np.random.default_rng(0)
+    for _ in range(12):
+        r, i = rng.integers(0, H.shape[0]), rng.integers(0, H.shape[1])
+        Hp, Hm = H.copy(), H.copy(); Hp[r, i] += eps; Hm[r, i] -= eps
+        assert math.isclose((frozen(Hp, W) - frozen(Hm, W)) / (2 * eps), dH[r, i], rel_tol=1e-6, abs_tol=1e-10)
+        v, j = rng.integers(0, W.shape[0]), rng.integers(0, W.shape[1])
+        Wp, Wm = W.copy(), W.copy(); Wp[v, j] += eps; Wm[v, j] -= eps
+        assert math.isclose((frozen(H, Wp) - frozen(H, Wm)) / (2 * eps), dW[v, j], rel_tol=1e-6, abs_tol=1e-10)
+    # each row of dz sums to zero (both softmaxes and the one-hot have unit mass): columns of dW summed over v vanish
+    assert np.allclose(dW.sum(axis=0), 0.0, atol=1e-14)
