@@ -251,6 +251,63 @@ int cat_conf_window(const float* conf_seq, int64_t L, const int64_t* block_start
                     int32_t K, float* conf_ext, void* cuda_stream);
 
 /*
+ * The full training loss of Section 3.3, Eq. 12: cross-entropy plus distillation from the target
+ * model, both under the CAT weight,
+ *     loss = (1/N) sum_r weight[r] * (beta * CE_r + KD_r),      KD_r = KL(p_t || q_r) = sum_v p_t[v] (log p_t[v] - log q_r[v]),
+ * q_r = softmax(H[r,:] W^T) the draft's distribution and p_t = softmax(Ht[t,:] Wt^T) the target's
+ * at the sequence position the row predicts.  The paper names the distillation loss without
+ * printing it; the forward KL at temperature 1 is this library's reading.  Draft row (block b,
+ * position k) refers to target position t = block_start[b] + k, so one row of target logits serves
+ * every draft row that predicts that position and the target GEMM covers L positions, not T rows.
+ * A row whose target position is outside [0, L) is an invalid row.  Gradients (weights constant,
+ * no gradient to the target side):
+ *     dz[r, v] = g * weight[r]/N * ((1 + beta) q_r[v] - beta [v == y_r] - p_t[v]),  dH = dz W,  dW = dz^T H.
+ * Confidences for the weights (Eq. 9): conf_ext if given; else, by desc->conf_source, the target's
+ * probability of the row's label (Eq. 9 as printed) or the draft's own.
+ *
+ * Works like cat_loss_fwd_bwd (row slabs, logits kept as fp16, three contractions) plus, per slab,
+ * a second vocabulary-chunked logits GEMM on the target side whose fp16 logits are kept for the
+ * slab.  bf16 inputs only (CAT_ERR_DTYPE otherwise).
+ */
+typedef enum { CAT_CONF_TARGET = 0, CAT_CONF_DRAFT = 1 } cat_conf_source;
+
+typedef struct {
+    int64_t L;            /* target positions = rows of Ht                                      */
+    int64_t d_t;          /* target hidden size (d_t % 8 == 0)                                  */
+    int64_t ldHt, ldWt;   /* row pitches of Ht and Wt in elements (>= d_t, multiples of 8)      */
+    float   beta;         /* weight of the cross-entropy term in Eq. 12 (the paper trains with 0.1) */
+    int32_t conf_source;  /* cat_conf_source, used when conf_ext == NULL                        */
+} cat_kd_desc;
+
+/*
+ * Scratch bytes of cat_kd_loss_fwd_bwd for this problem (0 if anything is invalid).  Needs the
+ * block starts because the target slab is sized by the widest range of positions one draft slab
+ * refers to.  `block_start_host`: HOST pointer, T/K entries, non-decreasing.
+ */
+size_t cat_kd_workspace_bytes(const cat_shape* shape, const cat_kd_desc* desc, const int64_t* block_start_host);
+
+/*
+ *   shape, H, W, labels, valid, grad_loss, lse, conf, weight, stats, dH, dW, accumulate_dW:
+ *                     as in cat_loss_fwd_bwd (device pointers)
+ *   desc              target-side sizes, beta, confidence source                        (host, in)
+ *   Ht, Wt            [L, d_t], [V, d_t] bf16 target hidden states and target LM head    (device, in)
+ *   block_start_host  [T/K] int64, HOST pointer, non-decreasing: sequence position of each block's
+ *                     first drafted token.  Copied to the device inside the call (one
+ *                     cudaMemcpyAsync on the stream); the caller may reuse it on return.
+ *   conf_ext          [T] fp32 or NULL                                                   (device, in)
+ *   loss              [3] fp32: total, its cross-entropy part (1/N) sum w CE, its distillation
+ *                     part (1/N) sum w KD; total = beta * loss[1] + loss[2]              (device, out)
+ *   workspace         at least cat_kd_workspace_bytes(...) bytes, 256-byte aligned       (device, scratch)
+ * Returns CAT_OK or a negative cat_status (CAT_ERR_SHAPE also for unsorted block starts).
+ */
+int cat_kd_loss_fwd_bwd(const cat_shape* shape, const cat_kd_desc* desc, const void* H, const void* W,
+                        const int64_t* labels, const uint8_t* valid, const void* Ht, const void* Wt,
+                        const int64_t* block_start_host, const float* conf_ext, const float* grad_loss,
+                        float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                        void* dH, void* dW, int accumulate_dW,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Number of kernels of this library that the given pass (0 = cat_loss_fwd, 1 = cat_loss_bwd,
  * 2 = cat_loss_fwd_bwd) launches for this shape: the logits GEMM, the per-row kernels and the final reduction in
  * the forward pass; one set-up kernel plus three GEMMs per vocabulary slab in the backward

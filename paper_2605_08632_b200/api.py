@@ -33,6 +33,8 @@ class CatLoss:
         self.ws_fwd = torch.empty(nf, dtype=torch.uint8, device=dev)
         self.ws_bwd = torch.empty(nb, dtype=torch.uint8, device=dev)
         self._ws_fused = None
+        self._ws_kd = None
+        self.loss3 = None
         self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
         self.lse = torch.empty(T, dtype=torch.float32, device=dev)
         self.conf = torch.empty(T, dtype=torch.float32, device=dev)
@@ -66,6 +68,26 @@ class CatLoss:
         out = torch.empty(self.T // self.K, dtype=torch.float32, device=self.loss.device)
         B.cat_accept_len(self.shape, self.conf, self.weight, out)
         return out
+
+    def kd_forward_backward(self, H, W, labels, valid, Ht, Wt, block_start_host, beta, conf_source=B.CAT_CONF_TARGET,
+                            conf_ext=None, grad_loss=None, accumulate_dW=False):
+        """cat_kd_loss_fwd_bwd: Eq. 12, CAT-weighted cross-entropy + distillation from the target head.
+        Returns (loss3, dH, dW) with loss3 = [total, cross-entropy part, distillation part]."""
+        desc = B.make_kd_desc(Ht.shape[0], Ht.shape[1], float(beta), conf_source, ldHt=Ht.stride(0), ldWt=Wt.stride(0))
+        n = B.cat_kd_workspace_bytes(self.shape, desc, block_start_host)
+        if n == 0:
+            raise ValueError("invalid problem for cat_kd_loss_fwd_bwd")
+        if self._ws_kd is None or self._ws_kd.numel() < n:
+            self._ws_kd = torch.empty(n, dtype=torch.uint8, device=self.loss.device)
+        if self.loss3 is None:
+            self.loss3 = torch.zeros(3, dtype=torch.float32, device=self.loss.device)
+        B.cat_kd_loss_fwd_bwd(self.shape, desc, H, W, labels, valid, Ht, Wt, block_start_host, conf_ext, grad_loss,
+                              self.loss3, self.lse, self.conf, self.weight, self.stats, self.dH, self.dW, accumulate_dW,
+                              self._ws_kd)
+        return self.loss3, self.dH, self.dW
+
+    def kd_status(self) -> int:
+        return int(self._ws_kd[:4].view(torch.int32).item())
 
     def fused_status(self) -> int:
         return int(self._ws_fused[:4].view(torch.int32).item())

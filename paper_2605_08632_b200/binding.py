@@ -30,6 +30,14 @@ class cat_stats(ctypes.Structure):
                 ("est_accept_len", ctypes.c_float), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+class cat_kd_desc(ctypes.Structure):
+    _fields_ = [("L", ctypes.c_int64), ("d_t", ctypes.c_int64), ("ldHt", ctypes.c_int64), ("ldWt", ctypes.c_int64),
+                ("beta", ctypes.c_float), ("conf_source", ctypes.c_int32)]
+
+
+CAT_CONF_TARGET, CAT_CONF_DRAFT = 0, 1
+
+
 class CatError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -66,6 +74,10 @@ def lib() -> ctypes.CDLL:
         L.cat_conf_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 6 + [vp, sz, vp]
         L.cat_conf_window.restype = ctypes.c_int
         L.cat_conf_window.argtypes = [vp, ctypes.c_int64, vp, ctypes.c_int64, ctypes.c_int32, vp, vp]
+        L.cat_kd_workspace_bytes.restype = sz
+        L.cat_kd_workspace_bytes.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc), vp]
+        L.cat_kd_loss_fwd_bwd.restype = ctypes.c_int
+        L.cat_kd_loss_fwd_bwd.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc)] + [vp] * 16 + [ctypes.c_int, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -156,6 +168,32 @@ def cat_conf_window(conf_seq, L, block_start, n_blocks, K, conf_ext) -> None:
     rc = lib().cat_conf_window(_ptr(conf_seq), int(L), _ptr(block_start), int(n_blocks), int(K), _ptr(conf_ext), _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_conf_window")
+
+
+def make_kd_desc(L, d_t, beta, conf_source=CAT_CONF_TARGET, ldHt=None, ldWt=None) -> cat_kd_desc:
+    return cat_kd_desc(L, d_t, d_t if ldHt is None else ldHt, d_t if ldWt is None else ldWt, beta, conf_source)
+
+
+def _host_i64(t):
+    """Host pointer of a contiguous int64 CPU tensor (block starts are read on the host)."""
+    if t.device.type != "cpu" or t.dtype != torch.int64 or not t.is_contiguous():
+        raise TypeError("block_start must be a contiguous int64 CPU tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def cat_kd_workspace_bytes(shape, desc, block_start_host) -> int:
+    return int(lib().cat_kd_workspace_bytes(ctypes.byref(shape), ctypes.byref(desc), _host_i64(block_start_host)))
+
+
+def cat_kd_loss_fwd_bwd(shape, desc, H, W, labels, valid, Ht, Wt, block_start_host, conf_ext, grad_loss, loss, lse, conf,
+                        weight, stats, dH, dW, accumulate_dW, workspace) -> None:
+    rc = lib().cat_kd_loss_fwd_bwd(ctypes.byref(shape), ctypes.byref(desc), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid),
+                                   _ptr(Ht), _ptr(Wt), _host_i64(block_start_host), _ptr(conf_ext), _ptr(grad_loss),
+                                   _ptr(loss), _ptr(lse), _ptr(conf), _ptr(weight), _ptr(stats), _ptr(dH), _ptr(dW),
+                                   int(bool(accumulate_dW)), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_kd_loss_fwd_bwd")
 
 
 def read_stats(stats_tensor: torch.Tensor) -> cat_stats:

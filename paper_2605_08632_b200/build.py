@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libcat_loss.so")
 SOURCES = [os.path.join(CSRC, "cat_api.cu")]
-HEADERS = [os.path.join(CSRC, f) for f in ("ptx.cuh", "tc_gemm.cuh", "simt.cuh", "rowops.cuh")] + [
+HEADERS = [os.path.join(CSRC, f) for f in ("ptx.cuh", "tc_gemm.cuh", "simt.cuh", "rowops.cuh", "kd.cuh")] + [
     os.path.join(os.path.dirname(PKG_DIR), "include", "cat_loss.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-cudart", "static", "-shared", "-Xcompiler", "-fPIC"]

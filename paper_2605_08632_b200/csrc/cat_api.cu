@@ -14,6 +14,7 @@
 
 #include <mutex>
 
+#include "kd.cuh"
 #include "rowops.cuh"
 #include "simt.cuh"
 #include "tc_gemm.cuh"
@@ -201,6 +202,80 @@ FusedPlan plan_fused(const cat_shape* s) {
     return p;
 }
 
+// Distillation side of cat_kd_loss_fwd_bwd: what one call needs beyond the fused plan.
+struct KdArgs {
+    const cat_kd_desc* desc;
+    const void* Ht;
+    const void* Wt;
+    const int64_t* block_start_host;
+    const float* user_conf_ext;
+};
+
+inline long long clampll(long long x, long long lo, long long hi) { return x < lo ? lo : (x > hi ? hi : x); }
+
+// Target positions [lo, lo + span) that the draft rows [r0, r0 + rws) refer to (block starts are sorted).
+void slab_target_range(const int64_t* start, long long r0, long long rws, int K, long long L, long long* lo, long long* span) {
+    const long long b0 = r0 / K, b1 = (r0 + rws) / K;       // slabs hold whole blocks
+    const long long a = clampll(start[b0], 0, L), b = clampll(start[b1 - 1] + K, 0, L);
+    *lo = a;
+    *span = b > a ? b - a : 0;
+}
+
+struct KdPlan {
+    long long Ls_max;       // most target positions any draft slab refers to
+    int S_t_max;            // most vocabulary splits of a target slab GEMM
+    size_t off_start, off_valid_eff, off_neg_labels, off_zt_label_row, off_conf_dev, off_kd_row, off_part_m_t, off_part_l_t,
+        off_zt_label_t, off_lse_t, off_conf_t, off_weight_t, off_partials_t, off_zt, total;
+};
+
+int check_kd(const cat_shape* s, const cat_kd_desc* k, const int64_t* start) {
+    if (!k || !start) return CAT_ERR_NULL;
+    if (s->in_dtype != CAT_BF16) return CAT_ERR_DTYPE;
+    if (k->L <= 0 || k->L >= (1ll << 31) || k->d_t <= 0 || k->d_t > 65536 || k->ldHt < k->d_t || k->ldWt < k->d_t) return CAT_ERR_SHAPE;
+    if (k->d_t % 8 != 0 || k->ldHt % 8 != 0 || k->ldWt % 8 != 0) return CAT_ERR_ALIGN;
+    if (!(k->beta >= 0.f && k->beta <= 3.0e38f)) return CAT_ERR_SHAPE;
+    if (k->conf_source != CAT_CONF_TARGET && k->conf_source != CAT_CONF_DRAFT) return CAT_ERR_SHAPE;
+    const long long nb = s->T / s->K;
+    for (long long b = 0; b + 1 < nb; ++b)
+        if (start[b] > start[b + 1]) return CAT_ERR_SHAPE;          // block starts must be sorted
+    if (start[0] < -(1ll << 40) || start[nb - 1] > (1ll << 40)) return CAT_ERR_SHAPE;
+    return CAT_OK;
+}
+
+KdPlan plan_kd(const cat_shape* s, const FusedPlan& fp, const cat_kd_desc* k, const int64_t* start, size_t base) {
+    KdPlan p;
+    p.Ls_max = 1;
+    p.S_t_max = 1;
+    for (long long r0 = 0; r0 < s->T; r0 += fp.Ts) {
+        const long long rws = (s->T - r0) < fp.Ts ? (s->T - r0) : fp.Ts;
+        long long lo, span;
+        slab_target_range(start, r0, rws, s->K, k->L, &lo, &span);
+        if (span > p.Ls_max) p.Ls_max = span;
+        if (span > 0) {
+            const int S = fwd_splits(span, s->V);
+            if (S > p.S_t_max) p.S_t_max = S;
+        }
+    }
+    const size_t Ls = static_cast<size_t>(p.Ls_max), T = static_cast<size_t>(s->T);
+    size_t off = align256(base);
+    p.off_start = off;        off = align256(off + sizeof(long long) * (T / s->K));
+    p.off_valid_eff = off;    off = align256(off + T);
+    p.off_neg_labels = off;   off = align256(off + sizeof(long long) * Ls);
+    p.off_zt_label_row = off; off = align256(off + sizeof(float) * T);
+    p.off_conf_dev = off;     off = align256(off + sizeof(float) * T);
+    p.off_kd_row = off;       off = align256(off + sizeof(float) * T);
+    p.off_part_m_t = off;     off = align256(off + sizeof(float) * p.S_t_max * Ls);
+    p.off_part_l_t = off;     off = align256(off + sizeof(float) * p.S_t_max * Ls);
+    p.off_zt_label_t = off;   off = align256(off + sizeof(float) * Ls);
+    p.off_lse_t = off;        off = align256(off + sizeof(float) * Ls);
+    p.off_conf_t = off;       off = align256(off + sizeof(float) * Ls);
+    p.off_weight_t = off;     off = align256(off + sizeof(float) * Ls);
+    p.off_partials_t = off;   off = align256(off + sizeof(rows::CtaPartial) * static_cast<size_t>(cdiv(p.Ls_max, rows::ROW_THREADS)));
+    p.off_zt = off;           off = align256(off + 2 * Ls * static_cast<size_t>(fp.ldz));
+    p.total = off;
+    return p;
+}
+
 // ------------------------------------------------------------------------------ device / driver
 int check_device(int* sm_count) {
     int dev = 0;
@@ -315,6 +390,218 @@ tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int b
     s.n_items = s.num_m_tiles * s.n_groups;
     return s;
 }
+
+// Forward + backward over row slabs with the slab's logits kept (cat_loss_fwd_bwd); with `kd` also the
+// distillation term of Eq. 12 (cat_kd_loss_fwd_bwd): per slab a second logits GEMM on the target
+// side, the target confidences of Eq. 9, and a dz that carries both terms.
+int fused_core(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid_in,
+               const float* conf_ext_in, const float* grad_loss, float* loss, float* lse, float* conf, float* weight,
+               cat_stats* stats, void* dH, void* dW, int accumulate_dW, void* workspace, size_t workspace_bytes,
+               void* cuda_stream, const KdArgs* kd) {
+    if (!shape || !H || !W || !labels || !loss || !lse || !conf || !weight || !dH || !dW) return CAT_ERR_NULL;
+    const int sc = check_shape(shape);
+    if (sc != CAT_OK) return sc;
+    const uint8_t* valid = valid_in;
+    const float* conf_ext = conf_ext_in;
+    if (kd) {
+        const int kc = check_kd(shape, kd->desc, kd->block_start_host);
+        if (kc != CAT_OK) return kc;
+        if (!kd->Ht || !kd->Wt) return CAT_ERR_NULL;
+        if (misaligned(kd->Ht, 16) || misaligned(kd->Wt, 16)) return CAT_ERR_ALIGN;
+    }
+    if (shape->in_dtype != CAT_BF16) {
+        // fp32 path: forward then backward, sharing one workspace (the passes run back to back)
+        const size_t need = cat_loss_workspace_bytes(shape, 2);
+        if (!workspace || misaligned(workspace, 256) || workspace_bytes < need) return CAT_ERR_WORKSPACE;
+        const int rc = cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, workspace,
+                                    workspace_bytes, cuda_stream);
+        if (rc != CAT_OK) return rc;
+        return cat_loss_bwd(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace,
+                            workspace_bytes, cuda_stream);
+    }
+    if (misaligned(H, 16) || misaligned(W, 16) || misaligned(dH, 16) || misaligned(dW, 16) || misaligned(labels, 8) ||
+        misaligned(loss, 4) || misaligned(lse, 4) || misaligned(conf, 4) || misaligned(weight, 4) ||
+        (conf_ext && misaligned(conf_ext, 4)) || (grad_loss && misaligned(grad_loss, 4)) || (stats && misaligned(stats, 8)))
+        return CAT_ERR_ALIGN;
+    const FusedPlan plan = plan_fused(shape);
+    KdPlan kp;
+    memset(&kp, 0, sizeof(kp));
+    if (kd) kp = plan_kd(shape, plan, kd->desc, kd->block_start_host, plan.total);
+    if (!workspace || misaligned(workspace, 256) || workspace_bytes < (kd ? kp.total : plan.total)) return CAT_ERR_WORKSPACE;
+    int sm_count = 0;
+    const int dc = check_device(&sm_count);
+    if (dc != CAT_OK) return dc;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws);
+    float* scale = reinterpret_cast<float*>(ws + kScaleOffset);
+    float* part_m = reinterpret_cast<float*>(ws + plan.off_part_m);
+    float* part_l = reinterpret_cast<float*>(ws + plan.off_part_l);
+    float* z_label = reinterpret_cast<float*>(ws + plan.off_z_label);
+    float* row_ce = reinterpret_cast<float*>(ws + plan.off_row_ce);
+    rows::CtaPartial* partials = reinterpret_cast<rows::CtaPartial*>(ws + plan.off_partials);
+    void* zs = ws + plan.off_z;
+    float* dw_acc = reinterpret_cast<float*>(ws + plan.off_dw_acc);
+    const int T = static_cast<int>(shape->T), V = static_cast<int>(shape->V), d = static_cast<int>(shape->d);
+    const long long* y = reinterpret_cast<const long long*>(labels);
+    const __nv_bfloat16* Hb = static_cast<const __nv_bfloat16*>(H);
+
+    CUtensorMap tmW_k, tmW_mn;
+    if (tmap_b(&tmW_k, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
+    if (tmap_mn_major(&tmW_mn, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    // distillation: device copies / scratch of this call
+    long long* start_dev = nullptr;
+    unsigned char* valid_eff = nullptr;
+    float *zt_label_row = nullptr, *conf_dev = nullptr, *kd_row = nullptr;
+    CUtensorMap tmWt_k;
+    if (kd) {
+        start_dev = reinterpret_cast<long long*>(ws + kp.off_start);
+        valid_eff = ws + kp.off_valid_eff;
+        zt_label_row = reinterpret_cast<float*>(ws + kp.off_zt_label_row);
+        conf_dev = reinterpret_cast<float*>(ws + kp.off_conf_dev);
+        kd_row = reinterpret_cast<float*>(ws + kp.off_kd_row);
+        if (cudaMemcpyAsync(start_dev, kd->block_start_host, sizeof(long long) * (shape->T / shape->K), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemsetAsync(ws + kp.off_neg_labels, 0xFF, sizeof(long long) * kp.Ls_max, st) != cudaSuccess) {   // labels of -1: no label gather on the target side
+            cudaGetLastError();
+            return CAT_ERR_CUDA;
+        }
+        kd::prepare_kernel<<<static_cast<unsigned>(cdiv(T, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(
+            y, valid_in, start_dev, T, shape->K, V, kd->desc->L, valid_eff);
+        valid = valid_eff;      // from here on a row without a target position is an invalid row
+        if (tmap_b(&tmWt_k, kd->Wt, shape->V, kd->desc->d_t, kd->desc->ldWt) != CAT_OK) return CAT_ERR_CUDA;
+    }
+    rows::bwd_scale_kernel<<<1, 1024, 0, st>>>(y, valid, T, V, grad_loss, scale);
+    if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+
+    int cta0 = 0;
+    for (int sl = 0; sl < plan.n_slabs; ++sl) {
+        const long long r0 = static_cast<long long>(sl) * plan.Ts;
+        const long long rws = (shape->T - r0) < plan.Ts ? (shape->T - r0) : plan.Ts;
+        const bool first = sl == 0, last = sl == plan.n_slabs - 1;
+        const int S = fwd_splits(rws, shape->V);
+        const __nv_bfloat16* Hs = Hb + r0 * shape->ldH;
+        CUtensorMap tmH_k, tmH_mn, tmZ_k, tmZ_mn;
+        if (tmap_a(&tmH_k, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_mn_major(&tmH_mn, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_a(&tmZ_k, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
+        if (tmap_mn_major(&tmZ_mn, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
+        {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
+            const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);
+            tc::EpiFwdStore::Params ep;
+            ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
+            ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T;
+            ep.T = static_cast<int>(rws); ep.V = V;
+            const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        }
+        long long t_lo = 0, t_span = 0;
+        float* lse_t_slab = nullptr;
+        if (kd) {
+            // target side of this slab: logits of the positions its rows refer to (kept as fp16), their lse,
+            // and the target's confidence in each draft row's label (Eq. 9)
+            slab_target_range(kd->block_start_host, r0, rws, shape->K, kd->desc->L, &t_lo, &t_span);
+            lse_t_slab = reinterpret_cast<float*>(ws + kp.off_lse_t);
+            if (t_span > 0) {
+                const __nv_bfloat16* Hts = static_cast<const __nv_bfloat16*>(kd->Ht) + t_lo * kd->desc->ldHt;
+                CUtensorMap tmHt_k;
+                if (tmap_a(&tmHt_k, Hts, t_span, kd->desc->d_t, kd->desc->ldHt) != CAT_OK) return CAT_ERR_CUDA;
+                const int St = fwd_splits(t_span, shape->V);
+                const tc::Sched sched = make_sched(t_span, shape->V, kd->desc->d_t, St, band_tiles(kd->desc->d_t), 0);
+                tc::EpiFwdStore::Params ep;
+                ep.labels = reinterpret_cast<const long long*>(ws + kp.off_neg_labels);
+                ep.part_m = reinterpret_cast<float*>(ws + kp.off_part_m_t);
+                ep.part_l = reinterpret_cast<float*>(ws + kp.off_part_l_t);
+                ep.z_label = reinterpret_cast<float*>(ws + kp.off_zt_label_t);
+                ep.zs = reinterpret_cast<__half*>(ws + kp.off_zt); ep.ldz = plan.ldz; ep.part_stride = kp.Ls_max;
+                ep.T = static_cast<int>(t_span); ep.V = V;
+                const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmHt_k, tmWt_k, sched, ep, status, sm_count, st);
+                if (rc != CAT_OK) return rc;
+                rows::RowParams rp;
+                rp.part_m = ep.part_m; rp.part_l = ep.part_l; rp.z_label = ep.z_label; rp.labels = ep.labels;
+                rp.valid = nullptr; rp.conf_ext = nullptr;
+                rp.lse = lse_t_slab; rp.conf = reinterpret_cast<float*>(ws + kp.off_conf_t);
+                rp.weight = reinterpret_cast<float*>(ws + kp.off_weight_t); rp.row_ce = nullptr;
+                rp.partials = reinterpret_cast<rows::CtaPartial*>(ws + kp.off_partials_t); rp.part_stride = kp.Ls_max;
+                rp.T = static_cast<int>(t_span); rp.V = V; rp.K = 1; rp.S = St; rp.fixed_decay = 0; rp.gamma = 0.f;
+                rows::row_kernel<true><<<static_cast<unsigned>(cdiv(t_span, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(rp);
+            }
+            kd::target_conf_kernel<<<static_cast<unsigned>(cdiv(rws * 32, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(
+                static_cast<const __nv_bfloat16*>(kd->Ht), kd->desc->ldHt, static_cast<const __nv_bfloat16*>(kd->Wt), kd->desc->ldWt,
+                static_cast<int>(kd->desc->d_t), y, valid_eff, start_dev, shape->K, r0, static_cast<int>(rws), t_lo, lse_t_slab,
+                zt_label_row, conf_dev);
+            if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+            conf_ext = kd->user_conf_ext ? kd->user_conf_ext : (kd->desc->conf_source == CAT_CONF_TARGET ? conf_dev : nullptr);
+        }
+        int n_ctas;
+        {   // lse, confidence (Eq. 9), CAT weights (Eq. 10), loss partials of the slab's blocks
+            rows::RowParams rp;
+            rp.part_m = part_m + r0; rp.part_l = part_l + r0; rp.z_label = z_label + r0; rp.labels = y + r0;
+            rp.valid = valid ? valid + r0 : nullptr; rp.conf_ext = conf_ext ? conf_ext + r0 : nullptr;
+            rp.lse = lse + r0; rp.conf = conf + r0; rp.weight = weight + r0; rp.row_ce = row_ce + r0;
+            rp.partials = partials + cta0; rp.part_stride = T;
+            rp.T = static_cast<int>(rws); rp.V = V; rp.K = shape->K; rp.S = S;
+            rp.fixed_decay = shape->weight_mode == CAT_WEIGHT_FIXED_DECAY; rp.gamma = shape->decay_gamma;
+            if (plan.warp_scan) {
+                n_ctas = static_cast<int>(cdiv(rws, rows::ROW_THREADS));
+                rows::row_kernel<true><<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
+            } else {
+                n_ctas = static_cast<int>(cdiv(rws / shape->K, rows::ROW_THREADS));
+                rows::row_kernel<false><<<static_cast<unsigned>(cdiv(rws, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(rp);
+                rows::block_scan_kernel<<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
+            }
+            cta0 += n_ctas;
+        }
+        // logits -> dz in place
+        if (kd)
+            kd::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
+                zs, ws + kp.off_zt, plan.ldz, y, valid_eff, start_dev, shape->K, r0, t_lo, lse, lse_t_slab, weight, z_label,
+                zt_label_row, kd->desc->beta, kd_row, V);
+        else
+            rows::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
+                zs, plan.ldz, y + r0, valid ? valid + r0 : nullptr, lse + r0, weight + r0, z_label + r0, V);
+        if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+        {   // dH[r0 : r0 + rws, :] = (g/N) dz W : the whole vocabulary is contracted, written once
+            const tc::Sched sched = make_sched(rws, shape->d, shape->V, 0, 1, 1);
+            tc::EpiOut::Params ep;
+            memset(&ep, 0, sizeof(ep));
+            ep.alpha = scale; ep.M = static_cast<int>(rws); ep.N = d;
+            ep.out_bf16 = static_cast<__nv_bfloat16*>(dH) + r0 * shape->ldH; ep.ld_out = shape->ldH;
+            const int rc = launch_tc<0, 1, tc::EpiOut>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        }
+        {   // dW += (g/N) dz^T H[r0 : r0 + rws, :]
+            const tc::Sched sched = make_sched(shape->V, shape->d, rws, 0, 1, 1);
+            tc::EpiOut::Params ep;
+            memset(&ep, 0, sizeof(ep));
+            ep.alpha = scale; ep.M = V; ep.N = d;
+            if (shape->dW_dtype == CAT_F32) {
+                ep.out_f32 = static_cast<float*>(dW); ep.ld_out = shape->ldW;
+                if (!first || accumulate_dW) { ep.add_f32 = ep.out_f32; ep.ld_add = shape->ldW; }
+            } else if (!plan.dw_acc) {
+                ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW;
+                if (accumulate_dW) { ep.add_bf16 = ep.out_bf16; ep.ld_add = shape->ldW; }
+            } else {
+                // bf16 dW over several slabs: sum in fp32 scratch, round once at the end
+                if (first) {
+                    if (accumulate_dW) { ep.add_bf16 = static_cast<const __nv_bfloat16*>(dW); ep.ld_add = shape->ldW; }
+                } else {
+                    ep.add_f32 = dw_acc; ep.ld_add = shape->d;
+                }
+                if (last) { ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW; }
+                else { ep.out_f32 = dw_acc; ep.ld_out = shape->d; }
+            }
+            const int rc = launch_tc<1, 1, tc::EpiOut>(tmZ_mn, tmH_mn, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        }
+    }
+    rows::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(partials, cta0, T / shape->K, loss,
+                                                         reinterpret_cast<rows::StatsOut*>(stats), status);
+    if (kd) kd::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(kd_row, valid_eff, T, kd->desc->beta, loss);
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+}
+
 
 // cat_conf_fwd treats every sequence position as a draft block of its own (K = 1, Eq. 10 weights).
 cat_shape per_position_shape(const cat_shape* s) {
@@ -579,132 +866,26 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const
                      const float* conf_ext, const float* grad_loss, float* loss, float* lse, float* conf, float* weight,
                      cat_stats* stats, void* dH, void* dW, int accumulate_dW, void* workspace, size_t workspace_bytes,
                      void* cuda_stream) {
-    if (!shape || !H || !W || !labels || !loss || !lse || !conf || !weight || !dH || !dW) return CAT_ERR_NULL;
-    const int sc = check_shape(shape);
-    if (sc != CAT_OK) return sc;
-    if (shape->in_dtype != CAT_BF16) {
-        // fp32 path: forward then backward, sharing one workspace (the passes run back to back)
-        const size_t need = cat_loss_workspace_bytes(shape, 2);
-        if (!workspace || misaligned(workspace, 256) || workspace_bytes < need) return CAT_ERR_WORKSPACE;
-        const int rc = cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, workspace,
-                                    workspace_bytes, cuda_stream);
-        if (rc != CAT_OK) return rc;
-        return cat_loss_bwd(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace,
-                            workspace_bytes, cuda_stream);
-    }
-    if (misaligned(H, 16) || misaligned(W, 16) || misaligned(dH, 16) || misaligned(dW, 16) || misaligned(labels, 8) ||
-        misaligned(loss, 4) || misaligned(lse, 4) || misaligned(conf, 4) || misaligned(weight, 4) ||
-        (conf_ext && misaligned(conf_ext, 4)) || (grad_loss && misaligned(grad_loss, 4)) || (stats && misaligned(stats, 8)))
-        return CAT_ERR_ALIGN;
-    const FusedPlan plan = plan_fused(shape);
-    if (!workspace || misaligned(workspace, 256) || workspace_bytes < plan.total) return CAT_ERR_WORKSPACE;
-    int sm_count = 0;
-    const int dc = check_device(&sm_count);
-    if (dc != CAT_OK) return dc;
+    return fused_core(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW, accumulate_dW,
+                      workspace, workspace_bytes, cuda_stream, nullptr);
+}
 
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    int* status = reinterpret_cast<int*>(ws);
-    float* scale = reinterpret_cast<float*>(ws + kScaleOffset);
-    float* part_m = reinterpret_cast<float*>(ws + plan.off_part_m);
-    float* part_l = reinterpret_cast<float*>(ws + plan.off_part_l);
-    float* z_label = reinterpret_cast<float*>(ws + plan.off_z_label);
-    float* row_ce = reinterpret_cast<float*>(ws + plan.off_row_ce);
-    rows::CtaPartial* partials = reinterpret_cast<rows::CtaPartial*>(ws + plan.off_partials);
-    void* zs = ws + plan.off_z;
-    float* dw_acc = reinterpret_cast<float*>(ws + plan.off_dw_acc);
-    const int T = static_cast<int>(shape->T), V = static_cast<int>(shape->V), d = static_cast<int>(shape->d);
-    const long long* y = reinterpret_cast<const long long*>(labels);
-    const __nv_bfloat16* Hb = static_cast<const __nv_bfloat16*>(H);
+size_t cat_kd_workspace_bytes(const cat_shape* shape, const cat_kd_desc* desc, const int64_t* block_start_host) {
+    if (check_shape(shape) != CAT_OK || check_kd(shape, desc, block_start_host) != CAT_OK) return 0;
+    const FusedPlan fp = plan_fused(shape);
+    return plan_kd(shape, fp, desc, block_start_host, fp.total).total;
+}
 
-    CUtensorMap tmW_k, tmW_mn;
-    if (tmap_b(&tmW_k, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
-    if (tmap_mn_major(&tmW_mn, W, shape->V, shape->d, shape->ldW) != CAT_OK) return CAT_ERR_CUDA;
-    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
-    rows::bwd_scale_kernel<<<1, 1024, 0, st>>>(y, valid, T, V, grad_loss, scale);
-    if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
-
-    int cta0 = 0;
-    for (int sl = 0; sl < plan.n_slabs; ++sl) {
-        const long long r0 = static_cast<long long>(sl) * plan.Ts;
-        const long long rws = (shape->T - r0) < plan.Ts ? (shape->T - r0) : plan.Ts;
-        const bool first = sl == 0, last = sl == plan.n_slabs - 1;
-        const int S = fwd_splits(rws, shape->V);
-        const __nv_bfloat16* Hs = Hb + r0 * shape->ldH;
-        CUtensorMap tmH_k, tmH_mn, tmZ_k, tmZ_mn;
-        if (tmap_a(&tmH_k, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
-        if (tmap_mn_major(&tmH_mn, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
-        if (tmap_a(&tmZ_k, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
-        if (tmap_mn_major(&tmZ_mn, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
-        {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
-            const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);
-            tc::EpiFwdStore::Params ep;
-            ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
-            ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T;
-            ep.T = static_cast<int>(rws); ep.V = V;
-            const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
-            if (rc != CAT_OK) return rc;
-        }
-        int n_ctas;
-        {   // lse, confidence (Eq. 9), CAT weights (Eq. 10), loss partials of the slab's blocks
-            rows::RowParams rp;
-            rp.part_m = part_m + r0; rp.part_l = part_l + r0; rp.z_label = z_label + r0; rp.labels = y + r0;
-            rp.valid = valid ? valid + r0 : nullptr; rp.conf_ext = conf_ext ? conf_ext + r0 : nullptr;
-            rp.lse = lse + r0; rp.conf = conf + r0; rp.weight = weight + r0; rp.row_ce = row_ce + r0;
-            rp.partials = partials + cta0; rp.part_stride = T;
-            rp.T = static_cast<int>(rws); rp.V = V; rp.K = shape->K; rp.S = S;
-            rp.fixed_decay = shape->weight_mode == CAT_WEIGHT_FIXED_DECAY; rp.gamma = shape->decay_gamma;
-            if (plan.warp_scan) {
-                n_ctas = static_cast<int>(cdiv(rws, rows::ROW_THREADS));
-                rows::row_kernel<true><<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
-            } else {
-                n_ctas = static_cast<int>(cdiv(rws / shape->K, rows::ROW_THREADS));
-                rows::row_kernel<false><<<static_cast<unsigned>(cdiv(rws, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(rp);
-                rows::block_scan_kernel<<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
-            }
-            cta0 += n_ctas;
-        }
-        // logits -> dz in place
-        rows::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
-            zs, plan.ldz, y + r0, valid ? valid + r0 : nullptr, lse + r0, weight + r0, z_label + r0, V);
-        if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
-        {   // dH[r0 : r0 + rws, :] = (g/N) dz W : the whole vocabulary is contracted, written once
-            const tc::Sched sched = make_sched(rws, shape->d, shape->V, 0, 1, 1);
-            tc::EpiOut::Params ep;
-            memset(&ep, 0, sizeof(ep));
-            ep.alpha = scale; ep.M = static_cast<int>(rws); ep.N = d;
-            ep.out_bf16 = static_cast<__nv_bfloat16*>(dH) + r0 * shape->ldH; ep.ld_out = shape->ldH;
-            const int rc = launch_tc<0, 1, tc::EpiOut>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
-            if (rc != CAT_OK) return rc;
-        }
-        {   // dW += (g/N) dz^T H[r0 : r0 + rws, :]
-            const tc::Sched sched = make_sched(shape->V, shape->d, rws, 0, 1, 1);
-            tc::EpiOut::Params ep;
-            memset(&ep, 0, sizeof(ep));
-            ep.alpha = scale; ep.M = V; ep.N = d;
-            if (shape->dW_dtype == CAT_F32) {
-                ep.out_f32 = static_cast<float*>(dW); ep.ld_out = shape->ldW;
-                if (!first || accumulate_dW) { ep.add_f32 = ep.out_f32; ep.ld_add = shape->ldW; }
-            } else if (!plan.dw_acc) {
-                ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW;
-                if (accumulate_dW) { ep.add_bf16 = ep.out_bf16; ep.ld_add = shape->ldW; }
-            } else {
-                // bf16 dW over several slabs: sum in fp32 scratch, round once at the end
-                if (first) {
-                    if (accumulate_dW) { ep.add_bf16 = static_cast<const __nv_bfloat16*>(dW); ep.ld_add = shape->ldW; }
-                } else {
-                    ep.add_f32 = dw_acc; ep.ld_add = shape->d;
-                }
-                if (last) { ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW; }
-                else { ep.out_f32 = dw_acc; ep.ld_out = shape->d; }
-            }
-            const int rc = launch_tc<1, 1, tc::EpiOut>(tmZ_mn, tmH_mn, sched, ep, status, sm_count, st);
-            if (rc != CAT_OK) return rc;
-        }
-    }
-    rows::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(partials, cta0, T / shape->K, loss,
-                                                         reinterpret_cast<rows::StatsOut*>(stats), status);
-    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
+int cat_kd_loss_fwd_bwd(const cat_shape* shape, const cat_kd_desc* desc, const void* H, const void* W, const int64_t* labels,
+                        const uint8_t* valid, const void* Ht, const void* Wt, const int64_t* block_start_host,
+                        const float* conf_ext, const float* grad_loss, float* loss, float* lse, float* conf, float* weight,
+                        cat_stats* stats, void* dH, void* dW, int accumulate_dW, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    if (!desc || !block_start_host) return CAT_ERR_NULL;
+    KdArgs kd;
+    kd.desc = desc; kd.Ht = Ht; kd.Wt = Wt; kd.block_start_host = block_start_host; kd.user_conf_ext = conf_ext;
+    return fused_core(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW, accumulate_dW,
+                      workspace, workspace_bytes, cuda_stream, &kd);
 }
 
 int cat_accept_len(const cat_shape* shape, const float* conf, const float* weight, float* accept_len, void* cuda_stream) {
