@@ -154,6 +154,38 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * cat_loss_bwd that also tells the caller when each part of dW is final, so that a data-parallel
+ * trainer can start summing that part across GPUs while the rest is still being computed.  The
+ * backward pass walks the vocabulary in cat_loss_bwd_slabs() slabs; the rows
+ * [v_begin[i], v_begin[i+1]) of dW are complete once slab i's dW GEMM has run, and
+ * slab_events[i] is recorded on `cuda_stream` right after it.
+ *   slab_events  HOST array of n_events cudaEvent_t (as void*), created by the caller        (host, in)
+ *   n_events     must equal cat_loss_bwd_slabs(shape, NULL, 0)
+ * Everything else as cat_loss_bwd.  dH is final only when the whole call has run.
+ */
+int cat_loss_bwd_events(const cat_shape* shape, const void* H, const void* W,
+                        const int64_t* labels, const uint8_t* valid,
+                        const float* lse, const float* weight, const float* grad_loss,
+                        void* dH, void* dW, int accumulate_dW,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream,
+                        void* const* slab_events, int n_events);
+
+/*
+ * Number of vocabulary slabs of cat_loss_bwd for this shape (0 if the shape is invalid); if
+ * v_begin != NULL the first vocabulary row of up to `capacity` slabs is written to it (host
+ * array).  Slab i covers rows [v_begin[i], min(v_begin[i+1], V)).
+ */
+int cat_loss_bwd_slabs(const cat_shape* shape, int64_t* v_begin, int capacity);
+
+/*
+ * N of Eq. 11's batch mean: the number of rows with valid[r] != 0 (or valid == NULL) and
+ * 0 <= labels[r] < V, written to *n_valid (device int64).  A data-parallel caller sums it over
+ * its ranks to get the global normaliser before the backward pass.  Only T and V of `shape` are used.
+ */
+int cat_count_valid(const cat_shape* shape, const int64_t* labels, const uint8_t* valid, int64_t* n_valid,
+                    void* cuda_stream);
+
+/*
  * Forward and backward in one call, without recomputing the logits (same results as
  * cat_loss_fwd followed by cat_loss_bwd, within rounding).  Rows are processed in slabs of
  * whole draft blocks.  For each slab the logits GEMM also writes the slab's logits as fp16

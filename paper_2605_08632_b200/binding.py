@@ -74,6 +74,12 @@ def lib() -> ctypes.CDLL:
         L.cat_conf_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 6 + [vp, sz, vp]
         L.cat_conf_window.restype = ctypes.c_int
         L.cat_conf_window.argtypes = [vp, ctypes.c_int64, vp, ctypes.c_int64, ctypes.c_int32, vp, vp]
+        L.cat_loss_bwd_events.restype = ctypes.c_int
+        L.cat_loss_bwd_events.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 9 + [ctypes.c_int, vp, sz, vp, vp, ctypes.c_int]
+        L.cat_loss_bwd_slabs.restype = ctypes.c_int
+        L.cat_loss_bwd_slabs.argtypes = [ctypes.POINTER(cat_shape), vp, ctypes.c_int]
+        L.cat_count_valid.restype = ctypes.c_int
+        L.cat_count_valid.argtypes = [ctypes.POINTER(cat_shape), vp, vp, vp, vp]
         L.cat_kd_workspace_bytes.restype = sz
         L.cat_kd_workspace_bytes.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc), vp]
         L.cat_kd_loss_fwd_bwd.restype = ctypes.c_int
@@ -168,6 +174,37 @@ def cat_conf_window(conf_seq, L, block_start, n_blocks, K, conf_ext) -> None:
     rc = lib().cat_conf_window(_ptr(conf_seq), int(L), _ptr(block_start), int(n_blocks), int(K), _ptr(conf_ext), _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_conf_window")
+
+
+def cat_loss_bwd_slabs(shape) -> list:
+    """First vocabulary row of every slab of cat_loss_bwd, plus V at the end."""
+    n = int(lib().cat_loss_bwd_slabs(ctypes.byref(shape), None, 0))
+    if n <= 0:
+        raise ValueError("invalid shape for cat_loss_bwd")
+    arr = (ctypes.c_int64 * n)()
+    lib().cat_loss_bwd_slabs(ctypes.byref(shape), arr, n)
+    return list(arr) + [int(shape.V)]
+
+
+def cat_loss_bwd_events(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace, events) -> None:
+    """`events`: list of torch.cuda.Event, one per vocabulary slab; event i is recorded once rows
+    [slabs[i], slabs[i+1]) of dW are final."""
+    for e in events:          # torch creates the CUDA event lazily, on first record
+        if getattr(e, "cuda_event", 0) == 0:
+            e.record()
+    arr = (ctypes.c_void_p * len(events))(*[ctypes.c_void_p(e.cuda_event) for e in events])
+    rc = lib().cat_loss_bwd_events(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(lse), _ptr(weight),
+                                   _ptr(grad_loss), _ptr(dH), _ptr(dW), int(bool(accumulate_dW)), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream(),
+                                   arr, len(events))
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_loss_bwd_events")
+
+
+def cat_count_valid(shape, labels, valid, n_valid) -> None:
+    rc = lib().cat_count_valid(ctypes.byref(shape), _ptr(labels), _ptr(valid), _ptr(n_valid), _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_count_valid")
 
 
 def make_kd_desc(L, d_t, beta, conf_source=CAT_CONF_TARGET, ldHt=None, ldWt=None) -> cat_kd_desc:

@@ -737,9 +737,11 @@ int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int
     return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
 }
 
-int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
-                 const float* lse, const float* weight, const float* grad_loss, void* dH, void* dW, int accumulate_dW,
-                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+// cat_loss_bwd / cat_loss_bwd_events: `slab_events` (host array of cudaEvent_t, one per vocabulary
+// slab, or NULL) are recorded on the stream as soon as a slab's rows of dW are final.
+static int bwd_core(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                    const float* lse, const float* weight, const float* grad_loss, void* dH, void* dW, int accumulate_dW,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, void* const* slab_events) {
     if (!shape || !H || !W || !labels || !lse || !weight || !dH || !dW) return CAT_ERR_NULL;
     const int sc = check_shape(shape);
     if (sc != CAT_OK) return sc;
@@ -806,6 +808,7 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
                 }
                 const int rc = launch_tc<1, 1, tc::EpiOut>(tmDz_mn, tmH_mn, sched, ep, status, sm_count, st);
                 if (rc != CAT_OK) return rc;
+                if (slab_events && cudaEventRecord(static_cast<cudaEvent_t>(slab_events[sl]), st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
             }
             {   // dH (+)= (g/N) dz W[v0 : v0 + width, :]
                 const tc::Sched sched = make_sched(shape->T, shape->d, width, 0, 1, 1);
@@ -844,6 +847,7 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
                 if (accumulate_dW) { ep.add = ep.out; ep.ld_add = shape->ldW; }
                 const dim3 grid(static_cast<unsigned>(cdiv(w, simt::TM)), static_cast<unsigned>(op.n_groups));
                 simt::gemm_kernel<simt::MODE_OUT><<<grid, simt::THREADS, 0, st>>>(op, ep);
+                if (slab_events && cudaEventRecord(static_cast<cudaEvent_t>(slab_events[sl]), st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
             }
             {   // dH (+)= (g/N) dz W slice : A(m = r, k = v) = dz[r][v], B(k = v, n = i) = W[v][i]
                 simt::Operands op;
@@ -860,6 +864,42 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
         }
     }
     return CAT_OK;
+}
+
+int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                 const float* lse, const float* weight, const float* grad_loss, void* dH, void* dW, int accumulate_dW,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return bwd_core(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace, workspace_bytes,
+                    cuda_stream, nullptr);
+}
+
+int cat_loss_bwd_slabs(const cat_shape* shape, int64_t* v_begin, int capacity) {
+    if (check_shape(shape) != CAT_OK) return 0;
+    const BwdPlan plan = plan_bwd(shape);
+    for (int sl = 0; v_begin && sl < plan.n_slabs && sl < capacity; ++sl) v_begin[sl] = static_cast<int64_t>(sl) * plan.Vs;
+    return plan.n_slabs;
+}
+
+int cat_loss_bwd_events(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                        const float* lse, const float* weight, const float* grad_loss, void* dH, void* dW, int accumulate_dW,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream, void* const* slab_events, int n_events) {
+    if (!slab_events) return CAT_ERR_NULL;
+    if (check_shape(shape) != CAT_OK) return CAT_ERR_SHAPE;
+    if (n_events != plan_bwd(shape).n_slabs) return CAT_ERR_SHAPE;
+    for (int i = 0; i < n_events; ++i)
+        if (!slab_events[i]) return CAT_ERR_NULL;
+    return bwd_core(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace, workspace_bytes,
+                    cuda_stream, slab_events);
+}
+
+int cat_count_valid(const cat_shape* shape, const int64_t* labels, const uint8_t* valid, int64_t* n_valid, void* cuda_stream) {
+    if (!shape || !labels || !n_valid) return CAT_ERR_NULL;
+    if (shape->T <= 0 || shape->T >= (1ll << 31) || shape->V <= 0 || shape->V >= (1ll << 31)) return CAT_ERR_SHAPE;
+    if (misaligned(labels, 8) || misaligned(n_valid, 8)) return CAT_ERR_ALIGN;
+    rows::count_valid_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        reinterpret_cast<const long long*>(labels), valid, static_cast<int>(shape->T), static_cast<int>(shape->V),
+        reinterpret_cast<long long*>(n_valid));
+    return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
 }
 
 int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,

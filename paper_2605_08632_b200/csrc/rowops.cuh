@@ -232,6 +232,26 @@ __global__ void __launch_bounds__(1024) bwd_scale_kernel(const long long* labels
     }
 }
 
+// Single CTA: N = number of rows that take part (mask bit set and label inside [0, V)).
+__global__ void __launch_bounds__(1024) count_valid_kernel(const long long* labels, const unsigned char* valid, int T, int V,
+                                                           long long* n_out) {
+    __shared__ int sh[32];
+    int n = 0;
+    for (int r = threadIdx.x; r < T; r += 1024) {
+        const long long y = labels[r];
+        n += ((valid == nullptr || valid[r] != 0) && y >= 0 && y < V) ? 1 : 0;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) n += __shfl_down_sync(0xffffffffu, n, off);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long tot = 0;
+        for (int w = 0; w < 32; ++w) tot += sh[w];
+        *n_out = tot;
+    }
+}
+
 // Fused path: turn one row of stored fp16 logits into bf16 dz in place,
 //   dz[r, v] = weight_r * (exp(z[r, v] - lse_r) - [v == y_r]),
 // the label entry formed from the fp32 label logit.  One CTA per row, 16-byte vectors; columns
