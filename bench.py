@@ -112,7 +112,8 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override T (debug / profiling of a small case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--profile", choices=["fused", "two-call"], default=None,
+    ap.add_argument("--no-extras", action="store_true", help="skip the Eq. 12 (cross-entropy + distillation) timing")
+    ap.add_argument("--profile", choices=["fused", "two-call", "kd"], default=None,
                     help="run only that path for --warmup + --steps steps and exit (for ncu captures of a small case; prints no bench line)")
     args = ap.parse_args()
 
@@ -187,9 +188,17 @@ def main():
             return float(t.item())
         return ms
 
+    def kd_setup():
+        # Eq. 12 on the same batch: a Llama-3.1-8B-shaped target head (d_t = 4096) over the
+        # T/K + K - 1 sequence positions the batch's blocks refer to, beta = 0.1
+        ts = synth.make_target_side(batch, d_t=4096)
+        Ht, Wt = ts.Ht.to(dev), ts.Wt.to(dev)
+        return ts, (lambda: cl.kd_forward_backward(H, W, labels, valid, Ht, Wt, ts.block_start, 0.1))
+
     if args.profile:
+        fn = {"fused": step, "two-call": step_split}.get(args.profile) or kd_setup()[1]
         for _ in range(args.warmup + args.steps):
-            step() if args.profile == "fused" else step_split()
+            fn()
         torch.cuda.synchronize()
         print(json.dumps({"profile_run": args.profile, "T": T, "note": "not a benchmark value"}))
         return
@@ -232,6 +241,29 @@ def main():
     split_ms = reduce_max(ev0.elapsed_time(ev1)) / args.steps
     fwd_ms = statistics.mean(a.elapsed_time(b) for a, b in fwd_ev)
     assert cl.fwd_stats().device_status == 0 and cl.bwd_status() == 0, "device reported a timed-out wait"
+
+    # ---- Eq. 12 (CAT-weighted cross-entropy + distillation): four contractions, one of them on the target side
+    kd_info = None
+    if not args.no_extras and world == 1:
+        ts, kd_step = kd_setup()
+        for _ in range(3):
+            kd_step()
+        kd_steps = max(2, min(args.steps, 5))
+        barrier()
+        ev0.record(stream)
+        for _ in range(kd_steps):
+            kd_step()
+        ev1.record(stream)
+        barrier()
+        kd_ms = ev0.elapsed_time(ev1) / kd_steps
+        assert cl.kd_status() == 0, "device reported a timed-out wait"
+        kd_flops = 6.0 * T * spec.d * spec.V + 2.0 * ts.L * ts.d_t * spec.V
+        kd_info = {"what": "cat_kd_loss_fwd_bwd (Eq. 12): draft head as the workload, target head d_t=4096 over L=%d positions, beta=0.1" % ts.L,
+                   "ms_per_step": kd_ms, "value": T / (kd_ms * 1e-3), "unit": UNIT, "tflops_executed": kd_flops / (kd_ms * 1e-3) / 1e12,
+                   "steps": kd_steps}
+        del ts, kd_step
+        cl._ws_kd = None
+        torch.cuda.empty_cache()
 
     # ------------------------------------------------------------------ end to end with host buffers
     e2e = None
@@ -287,6 +319,7 @@ def main():
                      "peak_kind": f"{peaks['source']} sustained bf16 (kernel timed inside the step loop); burst {peaks['burst']}",
                      "timed": "cat_loss_fwd bracketed by CUDA events inside the two-call step loop (GEMM + two O(T) kernels, 0.2 %)",
                      "flops_per_launch": fwd_flops, "traffic": None},
+        "eq12_path": kd_info,
         "clocks": clocks, "e2e": e2e,
         "gpu_launches": None,
     }

@@ -64,6 +64,7 @@ __all__ = [
     "cat_dW_rows",
     "kd_target_rows",
     "cat_kd_forward_backward",
+    "cat_kd_rows",
 ]
 
 
@@ -331,15 +332,31 @@ def kd_target_rows(block_start, K: int, T: int) -> np.ndarray:
     return (st[:, None] + np.arange(K)[None, :]).reshape(-1)
 
 
+def _kd_row_stats(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows):
+    """Per-row pieces of Eq. 12 for the given draft rows: log-partitions of both sides,
+    CE = -log q_y, KD = sum_v p_v (log p_v - log q_v), and the label probabilities q_y, p_y."""
+    z = Hd[rows] @ Wd.T                              # draft logits
+    zt = Htd[tsafe[rows]] @ Wtd.T                    # target logits of each row's sequence position
+    _, _, lse = softmax_stats(z)
+    _, _, lse_t = softmax_stats(zt)
+    logq = z - lse[:, None]
+    logp = zt - lse_t[:, None]
+    p_t = np.exp(logp)
+    i = np.arange(len(rows))
+    yy = ysafe[rows]
+    return dict(lse=lse, lse_t=lse_t, ce=-logq[i, yy], kd=(p_t * (logp - logq)).sum(axis=1),
+                q_y=np.exp(logq[i, yy]), p_y=p_t[i, yy], q=np.exp(logq), p_t=p_t)
+
+
 def cat_kd_forward_backward(H, W, labels, valid, K: int, Ht, Wt, block_start, beta: float,
                             conf_source: str = "target", conf_ext=None, g: float = 1.0,
-                            fixed_decay_gamma=None, want_grads: bool = True):
+                            fixed_decay_gamma=None, want_grads: bool = True, row_chunk: int = 512):
     """loss = (1/N) sum_r s_r (beta * CE_r + KD_r)  (Eq. 12 summed over k and n), its parts, and
     the gradients of g * loss w.r.t. H and W with s held constant.
 
     Returns (fwd dict, dH, dW).  fwd has loss, loss_ce, loss_kd (each already divided by N, so
     loss = beta*loss_ce + loss_kd), lse, lse_t (per draft row), conf, weight, row_ce, row_kd,
-    eff_valid, n_valid, target_row.
+    eff_valid, n_valid, target_row.  Rows are processed in chunks only to bound memory.
     """
     Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
     Htd, Wtd = _as_f64(Ht), _as_f64(Wt)
@@ -352,24 +369,19 @@ def cat_kd_forward_backward(H, W, labels, valid, K: int, Ht, Wt, block_start, be
     ok = effective_valid(y, valid, V) & (t_row >= 0) & (t_row < L)
     ysafe = np.where(ok, y, 0)
     tsafe = np.where(ok, t_row, 0)
-
-    z = Hd @ Wd.T                                    # draft logits, all rows (small cases only)
-    zt = Htd[tsafe] @ Wtd.T                          # target logits of each draft row's position
-    _, _, lse = softmax_stats(z)
-    _, _, lse_t = softmax_stats(zt)
-    logq = z - lse[:, None]
-    logp = zt - lse_t[:, None]
-    p_t = np.exp(logp)
-    q = np.exp(logq)
-    rows = np.arange(T)
-    row_ce = np.where(ok, -logq[rows, ysafe], 0.0)                       # L^CE
-    row_kd = np.where(ok, (p_t * (logp - logq)).sum(axis=1), 0.0)        # L^KD = KL(p^t || q)
+    lse, lse_t, ce, kdv, q_y, p_y = (np.empty(T) for _ in range(6))
+    for r0 in range(0, T, row_chunk):
+        rows = np.arange(r0, min(T, r0 + row_chunk))
+        st = _kd_row_stats(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows)
+        lse[rows], lse_t[rows], ce[rows], kdv[rows], q_y[rows], p_y[rows] = st["lse"], st["lse_t"], st["ce"], st["kd"], st["q_y"], st["p_y"]
+    row_ce = np.where(ok, ce, 0.0)                                       # L^CE
+    row_kd = np.where(ok, kdv, 0.0)                                      # L^KD = KL(p^t || q)
     if conf_ext is not None:
         conf = np.where(ok, _as_f64(conf_ext), 1.0)
     elif conf_source == "target":
-        conf = np.where(ok, p_t[rows, ysafe], 1.0)                       # Eq. 9 as printed
+        conf = np.where(ok, p_y, 1.0)                                    # Eq. 9 as printed
     elif conf_source == "draft":
-        conf = np.where(ok, q[rows, ysafe], 1.0)
+        conf = np.where(ok, q_y, 1.0)
     else:
         raise ValueError("conf_source must be 'target' or 'draft'")
     w = cat_weights(conf, ok, K) if fixed_decay_gamma is None else fixed_decay_weights(fixed_decay_gamma, ok, K)
@@ -383,10 +395,43 @@ def cat_kd_forward_backward(H, W, labels, valid, K: int, Ht, Wt, block_start, be
     dH = np.zeros((T, d))
     dW = np.zeros((V, d))
     if N:
-        onehot = np.zeros((T, V))
-        onehot[rows, ysafe] = 1.0
         coef = np.where(ok, g * w / N, 0.0)
-        dz = coef[:, None] * (beta * (q - onehot) + (q - p_t))
-        dH = dz @ Wd
-        dW = dz.T @ Hd
+        for r0 in range(0, T, row_chunk):
+            rows = np.arange(r0, min(T, r0 + row_chunk))
+            dz = _kd_dz(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows, coef, beta)
+            dH[rows] = dz @ Wd
+            dW += dz.T @ Hd[rows]
     return fwd, dH, dW
+
+
+def _kd_dz(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows, coef, beta):
+    """dz of Eq. 12 for the given rows: coef_r * (beta (q - onehot) + (q - p_t))."""
+    st = _kd_row_stats(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows)
+    onehot = np.zeros_like(st["q"])
+    onehot[np.arange(len(rows)), ysafe[rows]] = 1.0
+    return coef[rows, None] * (beta * (st["q"] - onehot) + (st["q"] - st["p_t"]))
+
+
+def cat_kd_rows(H, W, labels, valid, K: int, Ht, Wt, block_start, beta: float, blocks, n_valid_total: int,
+                conf_source: str = "target", g: float = 1.0):
+    """Eq. 12 for a chosen set of whole draft blocks of a large batch (sampled full-size checks):
+    per-row lse, lse_t, conf, weight, CE, KD of those blocks' rows, and their dH rows, given N of
+    the whole batch.  Returns (rows, dict, dH_rows)."""
+    Hd, Wd, y = _as_f64(H), _as_f64(W), _as_i64(labels)
+    Htd, Wtd = _as_f64(Ht), _as_f64(Wt)
+    T, V, L = Hd.shape[0], Wd.shape[0], Htd.shape[0]
+    blocks = np.asarray(blocks, dtype=np.int64)
+    rows = (blocks[:, None] * K + np.arange(K)[None, :]).reshape(-1)
+    t_row = kd_target_rows(block_start, K, T)
+    ok_all = effective_valid(y, valid, V) & (t_row >= 0) & (t_row < L)
+    ysafe, tsafe = np.where(ok_all, y, 0), np.where(ok_all, t_row, 0)
+    st = _kd_row_stats(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows)
+    ok = ok_all[rows]
+    conf = np.where(ok, st["p_y"] if conf_source == "target" else st["q_y"], 1.0)
+    w = cat_weights(conf, ok, K)
+    coef = np.zeros(T)
+    coef[rows] = np.where(ok, g * w / n_valid_total, 0.0)
+    dz = _kd_dz(Hd, Wd, Htd, Wtd, ysafe, tsafe, rows, coef, beta)
+    out = dict(lse=st["lse"], lse_t=st["lse_t"], conf=conf, weight=w, row_ce=np.where(ok, st["ce"], 0.0),
+               row_kd=np.where(ok, st["kd"], 0.0), eff_valid=ok)
+    return rows, out, dz @ Wd

@@ -123,3 +123,39 @@ def test_config2_full_size_whole_forward_and_sampled_dW_rows():
         assert np.max(np.abs(out["lse"] - fwd["lse"])) <= tol["lse"] * np.abs(fwd["lse"]).max()
         assert rel_l2(out["dW"][vocab], dW_rows) <= tol["grad"], rel_l2(out["dW"][vocab], dW_rows)
         del out
+
+
+def test_config2_full_size_distillation_loss_sampled_blocks_and_invariants():
+    """cat_kd_loss_fwd_bwd (Eq. 12) at the benchmark's size: a Llama-3.1-8B-shaped target head
+    (d_t = 4096) over the T/K + K - 1 sequence positions the batch's blocks refer to."""
+    from paper_2605_08632_b200 import binding as B
+    batch = synth.make_batch(2)
+    ts = synth.make_target_side(batch, d_t=4096)
+    tol = TOL[torch.bfloat16]
+    beta = 0.1
+    dev = torch.device("cuda")
+    cl = CatLoss(batch.T, batch.d, batch.V, batch.K)
+    cl.kd_forward_backward(batch.H.to(dev), batch.W.to(dev), batch.labels.to(dev), batch.valid.to(dev), ts.Ht.to(dev),
+                           ts.Wt.to(dev), ts.block_start, beta)
+    torch.cuda.synchronize()
+    assert cl.kd_status() == 0 and cl.fwd_stats().device_status == 0
+    N = cl.fwd_stats().n_valid
+    assert N == batch.T
+    conf, weight = cl.conf.cpu().numpy(), cl.weight.cpu().numpy()
+    ok = np.ones(batch.T, bool)
+    assert weight.tobytes() == O.cat_weights_f32(conf, ok, batch.K).tobytes()        # bit-exact scan, all rows
+    dW = cl.dW.cpu().numpy().astype(np.float64)
+    assert np.abs(dW.sum(axis=0)).max() <= 2e-3 * np.abs(dW).sum(axis=0).max()       # every dz row sums to zero
+    blocks = np.unique(np.r_[np.random.default_rng(12).choice(batch.T // batch.K, 8, replace=False), 0, batch.T // batch.K - 1])
+    rows, out, dH_rows = O.cat_kd_rows(batch.H, batch.W, batch.labels, batch.valid, batch.K, ts.Ht, ts.Wt, ts.block_start, beta,
+                                       blocks, N)
+    assert np.max(np.abs(cl.lse.cpu().numpy()[rows] - out["lse"]) / np.maximum(1.0, np.abs(out["lse"]))) <= tol["lse"]
+    assert np.max(np.abs(conf[rows] - out["conf"]) / np.maximum(out["conf"], 1e-30)) <= tol["conf"]
+    assert np.all(np.abs(weight[rows] - out["weight"]) <= batch.K * tol["conf"] * out["weight"] + 1e-37)
+    assert out["conf"].max() > 0.3                                                   # later positions carry weight
+    g = cl.dH.float().cpu().numpy()[rows]
+    assert rel_l2(g, dH_rows) <= tol["grad"], rel_l2(g, dH_rows)
+    later = np.setdiff1d(np.arange(len(rows)), np.arange(0, len(rows), batch.K))
+    assert rel_l2(g[later], dH_rows[later]) <= 2 * tol["grad"]
+    tot, ce, kd = cl.loss3.cpu().numpy()
+    assert abs(tot - (beta * ce + kd)) <= 1e-6 * abs(tot) and kd > 0

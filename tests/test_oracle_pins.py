@@ -501,3 +501,13 @@ def test_eq12_gradients_match_finite_differences_with_frozen_weights():
         assert math.isclose((frozen(H, Wp) - frozen(H, Wm)) / (2 * eps), dW[v, j], rel_tol=1e-6, abs_tol=1e-10)
     # each row of dz sums to zero (both softmaxes and the one-hot have unit mass): columns of dW summed over v vanish
     assert np.allclose(dW.sum(axis=0), 0.0, atol=1e-14)
+
+
+def test_eq12_sampled_block_routine_agrees_with_the_whole_batch_routine():
+    H, W, y, valid, Ht, Wt, st = _kd_problem(35, B=9, K=4, masked=True)
+    fwd, dH, _ = O.cat_kd_forward_backward(H, W, y, valid, 4, Ht, Wt, st, 0.1, g=0.5, row_chunk=7)
+    rows, out, dH_rows = O.cat_kd_rows(H, W, y, valid, 4, Ht, Wt, st, 0.1, [0, 3, 8], fwd["n_valid"], g=0.5)
+    assert np.array_equal(rows, np.r_[0:4, 12:16, 32:36])
+    for key in ("lse", "lse_t", "conf", "weight", "row_ce", "row_kd"):
+        assert np.allclose(out[key], fwd[key][rows], rtol=1e-13, atol=0), key
+    assert np.allclose(dH_rows, dH[rows], rtol=1e-12, atol=1e-18)
