@@ -27,6 +27,11 @@ if ROOT not in sys.path:
 
 import torch
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the roofline kernel (forward logits GEMM,
+# CTA-pair build) on the bench workload, from the ncu capture summarised in
+# profiles/ncu_two_call_gemms_config2.md.  Valid for that kernel, workload and T only.
+ROOFLINE_TRAFFIC_BYTES = {("config2", 16384): 2848929024 + 21131008}
+
 METRIC = "cat_loss_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -274,25 +279,55 @@ def main():
         dH_h = torch.empty(T, spec.d, dtype=batch.torch_dtype).pin_memory()
         dW_h = torch.empty(spec.V, spec.d, dtype=torch.float32).pin_memory()
 
-        def e2e_step():
-            H.copy_(Hh, non_blocking=True); W.copy_(Wh, non_blocking=True)
-            labels.copy_(yh, non_blocking=True); valid.copy_(vh, non_blocking=True)
-            cl.forward_backward(H, W, labels, valid)
-            loss_h.copy_(cl.loss, non_blocking=True); dH_h.copy_(cl.dH, non_blocking=True); dW_h.copy_(cl.dW, non_blocking=True)
+        # Two slots of device inputs and outputs, three streams: while step i computes, the inputs of step
+        # i+1 arrive and the results of step i-1 leave.  Every step still copies its own inputs from pinned
+        # host memory and its own results (loss, dH, dW) back; the copies overlap other steps' compute.
+        cls = [cl, CatLoss(T, spec.d, spec.V, spec.K, dtype=batch.torch_dtype)]
+        ins = [(H, W, labels, valid), tuple(torch.empty_like(x) for x in (H, W, labels, valid))]
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        in_ready = [torch.cuda.Event() for _ in range(2)]
+        comp_done = [torch.cuda.Event() for _ in range(2)]
+        out_done = [torch.cuda.Event() for _ in range(2)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-        e2e_steps = max(2, min(args.steps, 5))
-        e2e_step()
+        def e2e_step(i):
+            k = i & 1
+            c, (Hd, Wd, yd, vd) = cls[k], ins[k]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(comp_done[k])            # the slot's previous step has read its inputs
+                Hd.copy_(Hh, non_blocking=True); Wd.copy_(Wh, non_blocking=True)
+                yd.copy_(yh, non_blocking=True); vd.copy_(vh, non_blocking=True)
+                in_ready[k].record(s_in)
+            stream.wait_event(in_ready[k])
+            stream.wait_event(out_done[k])               # the slot's previous results have left
+            c.forward_backward(Hd, Wd, yd, vd)
+            comp_done[k].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(comp_done[k])
+                loss_h.copy_(c.loss, non_blocking=True); dH_h.copy_(c.dH, non_blocking=True); dW_h.copy_(c.dW, non_blocking=True)
+                out_done[k].record(s_out)
+
+        e2e_steps = max(4, min(args.steps, 10))
+        for k in range(2):
+            comp_done[k].record(stream); out_done[k].record(stream)
+        e2e_step(0); e2e_step(1)
         barrier()
-        ev0.record(stream)
-        for _ in range(e2e_steps):
-            e2e_step()
-        ev1.record(stream)
+        t0.record(s_in)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        with torch.cuda.stream(s_out):
+            t1.record(s_out)
         barrier()
-        e_ms = reduce_max(ev0.elapsed_time(ev1))
+        e_ms = reduce_max(t0.elapsed_time(t1))
+        assert all(c.fused_status() == 0 for c in cls), "device reported a timed-out wait"
         h2d = sum(x.numel() * x.element_size() for x in (Hh, Wh, yh, vh))
         d2h = sum(x.numel() * x.element_size() for x in (loss_h, dH_h, dW_h))
         e2e = {"value": world * T / (e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps,
+               "how": "cat_loss_fwd_bwd through the binding; per step H2D of H, W, labels, valid from pinned memory and D2H of "
+                      "loss, dH, dW, double-buffered so that copies overlap the neighbouring steps' compute"}
+        del cls, ins
+        torch.cuda.empty_cache()
 
     if rank != 0:
         if world > 1:
@@ -318,7 +353,11 @@ def main():
                      "achieved": achieved, "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["sustained"],
                      "peak_kind": f"{peaks['source']} sustained bf16 (kernel timed inside the step loop); burst {peaks['burst']}",
                      "timed": "cat_loss_fwd bracketed by CUDA events inside the two-call step loop (GEMM + two O(T) kernels, 0.2 %)",
-                     "flops_per_launch": fwd_flops, "traffic": None},
+                     "flops_per_launch": fwd_flops,
+                     "traffic": (ROOFLINE_TRAFFIC_BYTES.get((f"config{args.config}", T))
+                                 if os.environ.get("CAT_LOSS_CTA_PAIR", "1") != "0" else None),
+                     "traffic_unit": "bytes per launch (ncu dram read + write); algorithmic bytes: W + H + partials = %d" % (
+                         spec.V * spec.d * 2 + T * spec.d * 2 + 2 * 4 * T * 128)},
         "eq12_path": kd_info,
         "clocks": clocks, "e2e": e2e,
         "gpu_launches": None,

@@ -787,7 +787,9 @@ static int bwd_core(const cat_shape* shape, const void* H, const void* W, const 
             if (tmap_a(&tmDz_k, dz, shape->T, width, plan.Vs) != CAT_OK) return CAT_ERR_CUDA;
             if (tmap_mn_major(&tmDz_mn, dz, shape->T, width, plan.Vs) != CAT_OK) return CAT_ERR_CUDA;
             {   // recompute the logits of this slab and turn them into dz
-                const tc::Sched sched = make_sched(shape->T, width, shape->d, 0, band_tiles(shape->d), 0);
+                // same item shape as the forward pass: (m-tile, run of vocabulary tiles), so the per-row state
+                // (label, lse, weight) is loaded once per run
+                const tc::Sched sched = make_sched(shape->T, width, shape->d, fwd_splits(shape->T, width), band_tiles(shape->d), 0);
                 tc::EpiDz::Params ep;
                 ep.labels = y; ep.valid = valid; ep.lse = lse; ep.weight = weight; ep.dz = dz; ep.ld = plan.Vs;
                 ep.T = T; ep.V = V; ep.v0 = static_cast<int>(v0);
