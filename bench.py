@@ -1,11 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the CAT loss hot path (fused LM head + CAT-weighted cross-entropy, fwd + bwd).
 
-One step = cat_loss_fwd + cat_loss_bwd over one synthetic draft-training batch of the
-Llama-3.2-1B-shaped head config (T=16384 rows in blocks of K=8, d=2048, V=128256, bf16).
+One step = the whole hot path, forward and backward (one cat_loss_fwd_bwd call), over one synthetic
+draft-training batch of the Llama-3.2-1B-shaped head config (T=16384 rows in blocks of K=8, d=2048,
+V=128256, bf16); the two-call form (cat_loss_fwd + cat_loss_bwd, logits recomputed) is timed beside it.
 Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
 metric with host (pinned) buffers, host<->device copies inside the timed region; `roofline`
-is the forward logits GEMM (2*T*d*V flops per launch) against the measured dense bf16 peak;
+is the GEMM with the largest share of the step, timed by events inside the timed steps, against
+the measured dense bf16 peak (`stages` has every stage; `roofline_fwd_two_call` the forward GEMM
+of the two-call path);
 `cpu_baseline` is the fp64 oracle timed on this machine's host cores on a bounded sample.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
@@ -27,10 +30,22 @@ if ROOT not in sys.path:
 
 import torch
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the roofline kernel (forward logits GEMM,
-# CTA-pair build) on the bench workload, from the ncu capture summarised in
-# profiles/ncu_two_call_gemms_config2.md.  Valid for that kernel, workload and T only.
-ROOFLINE_TRAFFIC_BYTES = {("config2", 16384): 2848929024 + 21131008}
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of a kernel (CTA-pair build) on the bench
+# workload, from the ncu captures summarised in profiles/ (ncu_full_fused_gemms_config2.md for the
+# first row slab of the one-call path, ncu_two_call_gemms_config2.md for the two-call forward).
+# Valid for that kernel, workload and T only; None for anything else.
+TRAFFIC_BYTES = {
+    ("config2", 16384, "logits"): 747252000 + 2388404000,
+    ("config2", 16384, "dH"): 8986855000 + 35412000,
+    ("config2", 16384, "dW"): 7414872000 + 1038830000,
+    ("config2", 16384, "fwd_two_call"): 2848929024 + 21131008,
+}
+STAGES = ("logits", "rows", "z_to_dz", "dH", "dW")
+STAGE_KERNEL = {
+    "logits": "tc::gemm_kernel<K-major,K-major,EpiFwdStore,pair> logits + softmax partials + fp16 logits store",
+    "dH": "tc::gemm_kernel<K-major,MN-major,EpiOut,pair> dH slab = dz W",
+    "dW": "tc::gemm_kernel<MN-major,MN-major,EpiOut,pair> dW += dz^T H",
+}
 
 METRIC = "cat_loss_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
@@ -218,9 +233,12 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     barrier()
+    # the timed steps go through cat_loss_fwd_bwd_events: the same kernels, plus an event recorded between
+    # stages, so that every kernel of the step is timed inside the timed region itself
+    stage_events = []
     ev0.record(stream)
     for i in range(args.steps):
-        step()
+        stage_events.append(cl.forward_backward_timed(H, W, labels, valid) if spec.dtype == "bf16" else step())
     ev1.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -337,6 +355,37 @@ def main():
     peaks = load_peaks()
     fwd_flops = 2.0 * T * spec.d * spec.V
     achieved = fwd_flops / (fwd_ms * 1e-3) / 1e12
+    pair = os.environ.get("CAT_LOSS_CTA_PAIR", "1") != "0"
+
+    # per-stage device times of the one-call path inside the timed region (averages over the timed steps)
+    stage_info, roofline = None, None
+    if spec.dtype == "bf16":
+        slabs = B.cat_loss_fused_slabs(cl.shape)
+        n_slabs = len(slabs) - 1
+        per = {st: [0.0] * n_slabs for st in STAGES}
+        other = 0.0
+        for evs in stage_events:
+            other += evs[0].elapsed_time(evs[1]) + evs[-2].elapsed_time(evs[-1])
+            for sl in range(n_slabs):
+                for j, st in enumerate(STAGES):
+                    per[st][sl] += evs[1 + 5 * sl + j].elapsed_time(evs[2 + 5 * sl + j])
+        for st in STAGES:
+            per[st] = [x / args.steps for x in per[st]]
+        stage_info = {"slab_rows": [slabs[i + 1] - slabs[i] for i in range(n_slabs)],
+                      "ms_per_launch": per, "ms_per_step": {st: sum(per[st]) for st in STAGES},
+                      "other_ms_per_step": other / args.steps}
+        # the roofline entry is the kernel with the largest share of the step, at its largest launch (first slab)
+        dom = max(("logits", "dH", "dW"), key=lambda st: sum(per[st]))
+        rows0 = slabs[1] - slabs[0]
+        flops0 = 2.0 * rows0 * spec.d * spec.V
+        ach = flops0 / (per[dom][0] * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": STAGE_KERNEL[dom], "launch": f"first row slab ({rows0} rows)",
+                    "achieved": ach, "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": ach / peaks["sustained"],
+                    "peak_kind": f"{peaks['source']} sustained bf16 (kernel timed inside the step loop); burst {peaks['burst']}",
+                    "timed": "CUDA events recorded by cat_loss_fwd_bwd_events around this launch, on the launching stream, in every timed step",
+                    "flops_per_launch": flops0, "share_of_step": sum(per[dom]) / ms_per_step,
+                    "traffic": TRAFFIC_BYTES.get((f"config{args.config}", T, dom)) if pair else None,
+                    "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"}
     tflops = value * flops_per_token / 1e12 / world
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -349,13 +398,13 @@ def main():
         "two_call_path": {"what": "cat_loss_fwd + cat_loss_bwd (logits recomputed, 8TdV executed)", "ms_per_step": split_ms,
                           "value": world * T / (split_ms * 1e-3), "tflops_6TdV_per_gpu": flops_per_token * T / (split_ms * 1e-3) / 1e12,
                           "fwd_ms": fwd_ms, "bwd_ms": split_ms - fwd_ms},
-        "roofline": {"bound": "tensor", "kernel": "tc::gemm_kernel<K-major,K-major,EpiFwd> (forward logits + online softmax)",
+        "roofline": roofline, "stages": stage_info,
+        "roofline_fwd_two_call": {"bound": "tensor", "kernel": "tc::gemm_kernel<K-major,K-major,EpiFwd,pair> (forward logits + online softmax)",
                      "achieved": achieved, "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["sustained"],
                      "peak_kind": f"{peaks['source']} sustained bf16 (kernel timed inside the step loop); burst {peaks['burst']}",
                      "timed": "cat_loss_fwd bracketed by CUDA events inside the two-call step loop (GEMM + two O(T) kernels, 0.2 %)",
                      "flops_per_launch": fwd_flops,
-                     "traffic": (ROOFLINE_TRAFFIC_BYTES.get((f"config{args.config}", T))
-                                 if os.environ.get("CAT_LOSS_CTA_PAIR", "1") != "0" else None),
+                     "traffic": TRAFFIC_BYTES.get((f"config{args.config}", T, "fwd_two_call")) if pair else None,
                      "traffic_unit": "bytes per launch (ncu dram read + write); algorithmic bytes: W + H + partials = %d" % (
                          spec.V * spec.d * 2 + T * spec.d * 2 + 2 * 4 * T * 128)},
         "eq12_path": kd_info,

@@ -209,6 +209,32 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W,
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * cat_loss_fwd_bwd with timing marks, for measuring the stages of the one-call path in place (the
+ * benchmark uses it to time the dominant GEMM inside its step loop).  The call walks the rows in
+ * cat_loss_fused_slabs() slabs; caller-owned events are recorded on `cuda_stream` in this order:
+ *     [0] start, [1] after the set-up kernel, then per slab s (base = 2 + 5 s):
+ *     [base] logits GEMM, [base+1] row kernel(s) (lse, Eq. 9, Eq. 10), [base+2] logits -> dz,
+ *     [base+3] dH GEMM, [base+4] dW GEMM; the last one after the final loss reduction.
+ *   stage_events  HOST array of n_events cudaEvent_t (as void*), created with timing enabled  (host, in)
+ *   n_events      must equal 5 * cat_loss_fused_slabs(shape, NULL, 0) + 3
+ * bf16 inputs only.  Everything else, results included, as cat_loss_fwd_bwd.
+ */
+int cat_loss_fwd_bwd_events(const cat_shape* shape, const void* H, const void* W,
+                            const int64_t* labels, const uint8_t* valid, const float* conf_ext,
+                            const float* grad_loss,
+                            float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
+                            void* dH, void* dW, int accumulate_dW,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream,
+                            void* const* stage_events, int n_events);
+
+/*
+ * Number of row slabs of cat_loss_fwd_bwd for this shape (0 if the shape is invalid or not bf16); if
+ * row_begin != NULL the first row of up to `capacity` slabs is written to it (host array).  Slab i
+ * covers rows [row_begin[i], min(row_begin[i+1], T)).
+ */
+int cat_loss_fused_slabs(const cat_shape* shape, int64_t* row_begin, int capacity);
+
+/*
  * cat_loss_fwd for callers that cannot hand over a workspace.  (The paper has no counterpart:
  * this is a packaging variant of the forward pass above, same arithmetic, same outputs.)
  *

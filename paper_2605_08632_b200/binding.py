@@ -74,6 +74,10 @@ def lib() -> ctypes.CDLL:
         L.cat_conf_fwd.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 6 + [vp, sz, vp]
         L.cat_conf_window.restype = ctypes.c_int
         L.cat_conf_window.argtypes = [vp, ctypes.c_int64, vp, ctypes.c_int64, ctypes.c_int32, vp, vp]
+        L.cat_loss_fwd_bwd_events.restype = ctypes.c_int
+        L.cat_loss_fwd_bwd_events.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 13 + [ctypes.c_int, vp, sz, vp, vp, ctypes.c_int]
+        L.cat_loss_fused_slabs.restype = ctypes.c_int
+        L.cat_loss_fused_slabs.argtypes = [ctypes.POINTER(cat_shape), vp, ctypes.c_int]
         L.cat_loss_bwd_events.restype = ctypes.c_int
         L.cat_loss_bwd_events.argtypes = [ctypes.POINTER(cat_shape)] + [vp] * 9 + [ctypes.c_int, vp, sz, vp, vp, ctypes.c_int]
         L.cat_loss_bwd_slabs.restype = ctypes.c_int
@@ -176,6 +180,37 @@ def cat_conf_window(conf_seq, L, block_start, n_blocks, K, conf_ext) -> None:
         raise CatError(rc, "cat_conf_window")
 
 
+def cat_loss_fused_slabs(shape) -> list:
+    """First row of every row slab of cat_loss_fwd_bwd, plus T at the end."""
+    n = int(lib().cat_loss_fused_slabs(ctypes.byref(shape), None, 0))
+    if n <= 0:
+        raise ValueError("invalid shape for cat_loss_fwd_bwd slabs")
+    arr = (ctypes.c_int64 * n)()
+    lib().cat_loss_fused_slabs(ctypes.byref(shape), arr, n)
+    return list(arr) + [int(shape.T)]
+
+
+def _event_array(events):
+    for e in events:          # torch creates the CUDA event lazily, on first record
+        if getattr(e, "cuda_event", 0) == 0:
+            e.record()
+    return (ctypes.c_void_p * len(events))(*[ctypes.c_void_p(e.cuda_event) for e in events])
+
+
+def cat_loss_fwd_bwd_events(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW,
+                            accumulate_dW, workspace, events) -> None:
+    """cat_loss_fwd_bwd that records `events` (torch.cuda.Event with enable_timing=True, 5 per row slab + 3)
+    between its stages."""
+    arr = _event_array(events)
+    rc = lib().cat_loss_fwd_bwd_events(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(conf_ext),
+                                       _ptr(grad_loss), _ptr(loss), _ptr(lse), _ptr(conf), _ptr(weight), _ptr(stats),
+                                       _ptr(dH), _ptr(dW), int(bool(accumulate_dW)), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream(),
+                                       arr, len(events))
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_loss_fwd_bwd_events")
+
+
 def cat_loss_bwd_slabs(shape) -> list:
     """First vocabulary row of every slab of cat_loss_bwd, plus V at the end."""
     n = int(lib().cat_loss_bwd_slabs(ctypes.byref(shape), None, 0))
@@ -189,10 +224,7 @@ def cat_loss_bwd_slabs(shape) -> list:
 def cat_loss_bwd_events(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace, events) -> None:
     """`events`: list of torch.cuda.Event, one per vocabulary slab; event i is recorded once rows
     [slabs[i], slabs[i+1]) of dW are final."""
-    for e in events:          # torch creates the CUDA event lazily, on first record
-        if getattr(e, "cuda_event", 0) == 0:
-            e.record()
-    arr = (ctypes.c_void_p * len(events))(*[ctypes.c_void_p(e.cuda_event) for e in events])
+    arr = _event_array(events)
     rc = lib().cat_loss_bwd_events(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(lse), _ptr(weight),
                                    _ptr(grad_loss), _ptr(dH), _ptr(dW), int(bool(accumulate_dW)), _ptr(workspace),
                                    workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream(),

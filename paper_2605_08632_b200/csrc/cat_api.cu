@@ -397,8 +397,11 @@ tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int b
 int fused_core(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid_in,
                const float* conf_ext_in, const float* grad_loss, float* loss, float* lse, float* conf, float* weight,
                cat_stats* stats, void* dH, void* dW, int accumulate_dW, void* workspace, size_t workspace_bytes,
-               void* cuda_stream, const KdArgs* kd) {
+               void* cuda_stream, const KdArgs* kd, void* const* marks = nullptr) {
     if (!shape || !H || !W || !labels || !loss || !lse || !conf || !weight || !dH || !dW) return CAT_ERR_NULL;
+    // optional timing marks (cat_loss_fwd_bwd_events): the next caller-owned event is recorded after each stage
+    int n_marked = 0;
+    auto mark = [&](cudaStream_t s) { if (marks) cudaEventRecord(static_cast<cudaEvent_t>(marks[n_marked++]), s); };
     const int sc = check_shape(shape);
     if (sc != CAT_OK) return sc;
     const uint8_t* valid = valid_in;
@@ -472,8 +475,10 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
         valid = valid_eff;      // from here on a row without a target position is an invalid row
         if (tmap_b(&tmWt_k, kd->Wt, shape->V, kd->desc->d_t, kd->desc->ldWt) != CAT_OK) return CAT_ERR_CUDA;
     }
+    mark(st);
     rows::bwd_scale_kernel<<<1, 1024, 0, st>>>(y, valid, T, V, grad_loss, scale);
     if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+    mark(st);
 
     int cta0 = 0;
     for (int sl = 0; sl < plan.n_slabs; ++sl) {
@@ -495,6 +500,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             ep.T = static_cast<int>(rws); ep.V = V;
             const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
+            mark(st);
         }
         long long t_lo = 0, t_span = 0;
         float* lse_t_slab = nullptr;
@@ -552,6 +558,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
                 rows::block_scan_kernel<<<n_ctas, rows::ROW_THREADS, 0, st>>>(rp);
             }
             cta0 += n_ctas;
+            mark(st);
         }
         // logits -> dz in place
         if (kd)
@@ -562,6 +569,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             rows::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
                 zs, plan.ldz, y + r0, valid ? valid + r0 : nullptr, lse + r0, weight + r0, z_label + r0, V);
         if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+        mark(st);
         {   // dH[r0 : r0 + rws, :] = (g/N) dz W : the whole vocabulary is contracted, written once
             const tc::Sched sched = make_sched(rws, shape->d, shape->V, 0, 1, 1);
             tc::EpiOut::Params ep;
@@ -570,6 +578,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             ep.out_bf16 = static_cast<__nv_bfloat16*>(dH) + r0 * shape->ldH; ep.ld_out = shape->ldH;
             const int rc = launch_tc<0, 1, tc::EpiOut>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
+            mark(st);
         }
         {   // dW += (g/N) dz^T H[r0 : r0 + rws, :]
             const tc::Sched sched = make_sched(shape->V, shape->d, rws, 0, 1, 1);
@@ -594,10 +603,12 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             }
             const int rc = launch_tc<1, 1, tc::EpiOut>(tmZ_mn, tmH_mn, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
+            mark(st);
         }
     }
     rows::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(partials, cta0, T / shape->K, loss,
                                                          reinterpret_cast<rows::StatsOut*>(stats), status);
+    mark(st);
     if (kd) kd::finalize_kernel<<<1, rows::ROW_THREADS, 0, st>>>(kd_row, valid_eff, T, kd->desc->beta, loss);
     return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
 }
@@ -873,6 +884,27 @@ int cat_loss_bwd(const cat_shape* shape, const void* H, const void* W, const int
                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return bwd_core(shape, H, W, labels, valid, lse, weight, grad_loss, dH, dW, accumulate_dW, workspace, workspace_bytes,
                     cuda_stream, nullptr);
+}
+
+int cat_loss_fused_slabs(const cat_shape* shape, int64_t* row_begin, int capacity) {
+    if (check_shape(shape) != CAT_OK || shape->in_dtype != CAT_BF16) return 0;
+    const FusedPlan plan = plan_fused(shape);
+    for (int sl = 0; row_begin && sl < plan.n_slabs && sl < capacity; ++sl) row_begin[sl] = static_cast<int64_t>(sl) * plan.Ts;
+    return plan.n_slabs;
+}
+
+int cat_loss_fwd_bwd_events(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
+                            const float* conf_ext, const float* grad_loss, float* loss, float* lse, float* conf, float* weight,
+                            cat_stats* stats, void* dH, void* dW, int accumulate_dW, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream, void* const* stage_events, int n_events) {
+    if (!stage_events) return CAT_ERR_NULL;
+    if (check_shape(shape) != CAT_OK) return CAT_ERR_SHAPE;
+    if (shape->in_dtype != CAT_BF16) return CAT_ERR_DTYPE;
+    if (n_events != 5 * plan_fused(shape).n_slabs + 3) return CAT_ERR_SHAPE;
+    for (int i = 0; i < n_events; ++i)
+        if (!stage_events[i]) return CAT_ERR_NULL;
+    return fused_core(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW, accumulate_dW,
+                      workspace, workspace_bytes, cuda_stream, nullptr, stage_events);
 }
 
 int cat_loss_bwd_slabs(const cat_shape* shape, int64_t* v_begin, int capacity) {

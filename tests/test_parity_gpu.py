@@ -174,6 +174,24 @@ def test_fused_fp32_inputs_and_determinism():
         assert a[key].tobytes() == b[key].tobytes(), key
 
 
+def test_fused_call_with_stage_events_gives_the_same_bits_and_ordered_times():
+    batch = synth.make_batch(41, T=1024, d=256, V=6000)
+    plain = run_gpu_fused(batch, slab_mib=4)
+    dev = torch.device("cuda")
+    cl = plain["obj"]
+    cl.dH.zero_(); cl.dW.zero_(); cl.lse.zero_()
+    evs = cl.forward_backward_timed(batch.H.to(dev), batch.W.to(dev), batch.labels.to(dev), batch.valid.to(dev))
+    torch.cuda.synchronize()
+    n_slabs = len(B.cat_loss_fused_slabs(cl.shape)) - 1
+    assert n_slabs >= 2 and len(evs) == 5 * n_slabs + 3
+    assert all(a.elapsed_time(b) >= 0.0 for a, b in zip(evs, evs[1:]))
+    for key, t in (("lse", cl.lse), ("weight", cl.weight), ("dH", cl.dH.float()), ("dW", cl.dW.float())):
+        assert t.cpu().numpy().tobytes() == plain[key].tobytes(), key
+    with pytest.raises(B.CatError):
+        B.cat_loss_fwd_bwd_events(cl.shape, batch.H.to(dev), batch.W.to(dev), batch.labels.to(dev), None, None, None, cl.loss,
+                                  cl.lse, cl.conf, cl.weight, cl.stats, cl.dH, cl.dW, False, cl._ws_fused, evs[:-1])
+
+
 def test_errors_on_gpu_box_leave_context_usable():
     s = B.make_shape(64, 128, 512, 8, B.CAT_BF16)
     x = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
