@@ -35,14 +35,11 @@ import torch
 # first row slab of the one-call path, ncu_two_call_gemms_config2.md for the two-call forward).
 # Valid for that kernel, workload and T only; None for anything else.
 TRAFFIC_BYTES = {
-    ("config2", 16384, "logits"): 747252000 + 2388404000,
-    ("config2", 16384, "dH"): 8986855000 + 35412000,
-    ("config2", 16384, "dW"): 7414872000 + 1038830000,
     ("config2", 16384, "fwd_two_call"): 2848929024 + 21131008,
 }
-STAGES = ("logits", "rows", "z_to_dz", "dH", "dW")
+STAGES = ("label_ref", "logits", "rows", "slab_prep", "dH", "dW")
 STAGE_KERNEL = {
-    "logits": "tc::gemm_kernel<K-major,K-major,EpiFwdStore,pair> logits + softmax partials + fp16 logits store",
+    "logits": "tc::gemm_kernel<K-major,K-major,EpiFwdExp,pair> logits + softmax partials + bf16 exp(z - ref) store",
     "dH": "tc::gemm_kernel<K-major,MN-major,EpiOut,pair> dH slab = dz W",
     "dW": "tc::gemm_kernel<MN-major,MN-major,EpiOut,pair> dW += dz^T H",
 }
@@ -368,7 +365,7 @@ def main():
             other += evs[0].elapsed_time(evs[1]) + evs[-2].elapsed_time(evs[-1])
             for sl in range(n_slabs):
                 for j, st in enumerate(STAGES):
-                    per[st][sl] += evs[1 + 5 * sl + j].elapsed_time(evs[2 + 5 * sl + j])
+                    per[st][sl] += evs[1 + len(STAGES) * sl + j].elapsed_time(evs[2 + len(STAGES) * sl + j])
         for st in STAGES:
             per[st] = [x / args.steps for x in per[st]]
         stage_info = {"slab_rows": [slabs[i + 1] - slabs[i] for i in range(n_slabs)],
@@ -394,7 +391,7 @@ def main():
         "tflops_6TdV_per_gpu": tflops,
         "frac_of_peak": {"measured_burst": tflops / peaks["burst"], "measured_sustained": tflops / peaks["sustained"],
                          "nominal_2250": tflops / 2250.0, "peaks": peaks["source"]},
-        "path": "cat_loss_fwd_bwd (logits kept as fp16 per row slab, 6TdV executed)",
+        "path": "cat_loss_fwd_bwd (softmax numerators kept as bf16 per row slab, 6TdV executed)",
         "two_call_path": {"what": "cat_loss_fwd + cat_loss_bwd (logits recomputed, 8TdV executed)", "ms_per_step": split_ms,
                           "value": world * T / (split_ms * 1e-3), "tflops_6TdV_per_gpu": flops_per_token * T / (split_ms * 1e-3) / 1e12,
                           "fwd_ms": fwd_ms, "bwd_ms": split_ms - fwd_ms},

@@ -188,15 +188,21 @@ int cat_count_valid(const cat_shape* shape, const int64_t* labels, const uint8_t
 /*
  * Forward and backward in one call, without recomputing the logits (same results as
  * cat_loss_fwd followed by cat_loss_bwd, within rounding).  Rows are processed in slabs of
- * whole draft blocks.  For each slab the logits GEMM also writes the slab's logits as fp16
- * (saturating at +-65504); once lse and the CAT weights of the slab's blocks are known
- * (Eq. 9, Eq. 10) the slab is turned in place into bf16
- * dz = weight * (exp(z - lse) - one-hot), the label entry taken from the fp32 label logit, and
- * feeds dH (written once per slab) and dW (accumulated over slabs in fp32).  Executed work is
- * the 6*T*d*V flops of the three contractions instead of 8*T*d*V; the price is one slab of
- * logits in the workspace (at most about slab_mib MiB, default 2560, and always at least two
- * slabs once T exceeds one slab unit, so the T x V logits never exist at once) and fp16 rounding of the stored logits
- * (relative 2^-11, i.e. about 1e-3 absolute on the logits of the synthetic configs).
+ * whole draft blocks.  For each slab the logits GEMM also writes e[r, v] = exp(z[r, v] - ref[r]) as
+ * bf16, the softmax numerators relative to a per-row reference fixed before the GEMM (the row's
+ * label logit, an fp32 dot product).  Once lse and the CAT weights of the slab's blocks are known
+ * (Eq. 9, Eq. 10), dz = weight * (softmax - one-hot) is a[r] * e'[r, v] with the per-row factor
+ * a[r] = weight[r] * exp(ref[r] - lse[r]) and e' = e with its label entry lowered by
+ * exp(lse[r] - ref[r]) (patched in place from the fp32 label logit): the dH GEMM applies a[r] in its
+ * epilogue, the dW GEMM takes a[r] * H[r, :] as its second operand, and no second pass over the slab
+ * is needed.  dH is written once per slab, dW accumulated over slabs in fp32.  Executed work is the
+ * 6*T*d*V flops of the three contractions instead of 8*T*d*V; the price is one slab of 16-bit values
+ * in the workspace (at most about slab_mib MiB, default 2560, and always at least two slabs once T
+ * exceeds one slab unit, so a T x V matrix never exists at once) and bf16 rounding of the stored
+ * numerators (relative 2^-9, the same as rounding dz to bf16).  The exponent z - ref is capped at
+ * 79.7 so that e stays finite for any input: only a row whose label is more than 79.7 nats below
+ * the row's largest logit (label probability under 1e-34) gets a damped gradient; its loss, lse and
+ * confidence are exact.
  * Arguments as in cat_loss_fwd and cat_loss_bwd; workspace of
  * cat_loss_workspace_bytes(shape, 2) bytes; cat_loss_launch_count(shape, 2) kernels.
  * For CAT_F32 inputs this runs the fp32 forward and backward passes back to back.
@@ -212,11 +218,12 @@ int cat_loss_fwd_bwd(const cat_shape* shape, const void* H, const void* W,
  * cat_loss_fwd_bwd with timing marks, for measuring the stages of the one-call path in place (the
  * benchmark uses it to time the dominant GEMM inside its step loop).  The call walks the rows in
  * cat_loss_fused_slabs() slabs; caller-owned events are recorded on `cuda_stream` in this order:
- *     [0] start, [1] after the set-up kernel, then per slab s (base = 2 + 5 s):
- *     [base] logits GEMM, [base+1] row kernel(s) (lse, Eq. 9, Eq. 10), [base+2] logits -> dz,
- *     [base+3] dH GEMM, [base+4] dW GEMM; the last one after the final loss reduction.
+ *     [0] start, [1] after the set-up kernel, then per slab s (base = 2 + 6 s):
+ *     [base] label-logit reference, [base+1] logits GEMM, [base+2] row kernel(s) (lse, Eq. 9, Eq. 10),
+ *     [base+3] per-row factor / label patch / scaled H rows, [base+4] dH GEMM, [base+5] dW GEMM;
+ *     the last one after the final loss reduction.
  *   stage_events  HOST array of n_events cudaEvent_t (as void*), created with timing enabled  (host, in)
- *   n_events      must equal 5 * cat_loss_fused_slabs(shape, NULL, 0) + 3
+ *   n_events      must equal 6 * cat_loss_fused_slabs(shape, NULL, 0) + 3
  * bf16 inputs only.  Everything else, results included, as cat_loss_fwd_bwd.
  */
 int cat_loss_fwd_bwd_events(const cat_shape* shape, const void* H, const void* W,

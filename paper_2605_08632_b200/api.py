@@ -64,12 +64,13 @@ class CatLoss:
 
     def forward_backward_timed(self, H, W, labels, valid=None, conf_ext=None, grad_loss=None, accumulate_dW=False):
         """cat_loss_fwd_bwd_events: same results as forward_backward; returns the stage events
-        (start, set-up, then per row slab: logits GEMM, row kernel, logits->dz, dH GEMM, dW GEMM; finalize)."""
+        (start, set-up, then per row slab: label reference, logits GEMM, row kernel, slab preparation,
+        dH GEMM, dW GEMM; finalize)."""
         if self._ws_fused is None:
             n = B.cat_loss_workspace_bytes(self.shape, 2)
             self._ws_fused = torch.empty(n, dtype=torch.uint8, device=self.loss.device)
         n_slabs = len(B.cat_loss_fused_slabs(self.shape)) - 1
-        events = [torch.cuda.Event(enable_timing=True) for _ in range(5 * n_slabs + 3)]
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(6 * n_slabs + 3)]
         B.cat_loss_fwd_bwd_events(self.shape, H, W, labels, valid, conf_ext, grad_loss, self.loss, self.lse, self.conf,
                                   self.weight, self.stats, self.dH, self.dW, accumulate_dW, self._ws_fused, events)
         return events

@@ -199,7 +199,7 @@ def _event_array(events):
 
 def cat_loss_fwd_bwd_events(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW,
                             accumulate_dW, workspace, events) -> None:
-    """cat_loss_fwd_bwd that records `events` (torch.cuda.Event with enable_timing=True, 5 per row slab + 3)
+    """cat_loss_fwd_bwd that records `events` (torch.cuda.Event with enable_timing=True, 6 per row slab + 3)
     between its stages."""
     arr = _event_array(events)
     rc = lib().cat_loss_fwd_bwd_events(ctypes.byref(shape), _ptr(H), _ptr(W), _ptr(labels), _ptr(valid), _ptr(conf_ext),

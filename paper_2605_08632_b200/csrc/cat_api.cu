@@ -148,7 +148,7 @@ struct FusedPlan {
     int n_row_ctas;        // per-row / per-block kernel CTAs summed over the slabs
     bool warp_scan;
     bool dw_acc;           // bf16 dW with several slabs: accumulate in an fp32 scratch copy
-    size_t off_part_m, off_part_l, off_z_label, off_row_ce, off_partials, off_z, off_dw_acc, total;
+    size_t off_part_m, off_part_l, off_z_label, off_row_ce, off_partials, off_ref, off_a, off_hs, off_z, off_dw_acc, total;
 };
 
 long long gcd_ll(long long a, long long b) { return b == 0 ? a : gcd_ll(b, a % b); }
@@ -195,6 +195,9 @@ FusedPlan plan_fused(const cat_shape* s) {
     p.off_z_label = off; off = align256(off + sizeof(float) * s->T);
     p.off_row_ce = off;  off = align256(off + sizeof(float) * s->T);
     p.off_partials = off; off = align256(off + sizeof(rows::CtaPartial) * p.n_row_ctas);
+    p.off_ref = off;     off = align256(off + sizeof(float) * s->T);                                  // reference of the stored exp(z - ref)
+    p.off_a = off;       off = align256(off + sizeof(float) * s->T);                                  // per-row factor of the backward
+    p.off_hs = off;      off = align256(off + 2 * static_cast<size_t>(p.Ts) * static_cast<size_t>(s->d));   // a[r] * H[r, :] of one slab
     p.off_z = off;       off = align256(off + 2 * static_cast<size_t>(p.Ts) * p.ldz);
     p.off_dw_acc = off;
     if (p.dw_acc) off = align256(off + sizeof(float) * static_cast<size_t>(s->V) * s->d);
@@ -446,6 +449,9 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
     rows::CtaPartial* partials = reinterpret_cast<rows::CtaPartial*>(ws + plan.off_partials);
     void* zs = ws + plan.off_z;
     float* dw_acc = reinterpret_cast<float*>(ws + plan.off_dw_acc);
+    float* ref = reinterpret_cast<float*>(ws + plan.off_ref);
+    float* a_row = reinterpret_cast<float*>(ws + plan.off_a);
+    __nv_bfloat16* h_scaled = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_hs);
     const int T = static_cast<int>(shape->T), V = static_cast<int>(shape->V), d = static_cast<int>(shape->d);
     const long long* y = reinterpret_cast<const long long*>(labels);
     const __nv_bfloat16* Hb = static_cast<const __nv_bfloat16*>(H);
@@ -492,13 +498,28 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
         if (tmap_mn_major(&tmH_mn, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_a(&tmZ_k, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_mn_major(&tmZ_mn, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
-        {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
+        if (kd) {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
             const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);
             tc::EpiFwdStore::Params ep;
             ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
-            ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T;
+            ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T; ep.ref = nullptr;
             ep.T = static_cast<int>(rws); ep.V = V;
             const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+            if (rc != CAT_OK) return rc;
+        } else {
+            // per-row reference (the label logit), then the logits GEMM: softmax partials + label logit,
+            // and exp(z - ref) kept as bf16 so that the backward needs no second pass over the slab
+            rows::label_ref_kernel<<<static_cast<unsigned>(cdiv(rws * 32, rows::ROW_THREADS)), rows::ROW_THREADS, 0, st>>>(
+                Hs, shape->ldH, static_cast<const __nv_bfloat16*>(W), shape->ldW, d, y + r0, valid ? valid + r0 : nullptr,
+                static_cast<int>(rws), V, ref + r0);
+            if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
+            mark(st);
+            const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);
+            tc::EpiFwdExp::Params ep;
+            ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
+            ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T; ep.ref = ref + r0;
+            ep.T = static_cast<int>(rws); ep.V = V;
+            const int rc = launch_tc<0, 0, tc::EpiFwdExp>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
             mark(st);
         }
@@ -520,7 +541,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
                 ep.part_m = reinterpret_cast<float*>(ws + kp.off_part_m_t);
                 ep.part_l = reinterpret_cast<float*>(ws + kp.off_part_l_t);
                 ep.z_label = reinterpret_cast<float*>(ws + kp.off_zt_label_t);
-                ep.zs = reinterpret_cast<__half*>(ws + kp.off_zt); ep.ldz = plan.ldz; ep.part_stride = kp.Ls_max;
+                ep.zs = reinterpret_cast<__half*>(ws + kp.off_zt); ep.ldz = plan.ldz; ep.part_stride = kp.Ls_max; ep.ref = nullptr;
                 ep.T = static_cast<int>(t_span); ep.V = V;
                 const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmHt_k, tmWt_k, sched, ep, status, sm_count, st);
                 if (rc != CAT_OK) return rc;
@@ -560,14 +581,18 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             cta0 += n_ctas;
             mark(st);
         }
-        // logits -> dz in place
-        if (kd)
+        if (kd) {
+            // both slabs of logits -> dz in place
             kd::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
                 zs, ws + kp.off_zt, plan.ldz, y, valid_eff, start_dev, shape->K, r0, t_lo, lse, lse_t_slab, weight, z_label,
                 zt_label_row, kd->desc->beta, kd_row, V);
-        else
-            rows::z_to_dz_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
-                zs, plan.ldz, y + r0, valid ? valid + r0 : nullptr, lse + r0, weight + r0, z_label + r0, V);
+        } else {
+            // dz = a[r] * e' : per-row factor, patched label entry, and the scaled copy of the slab's H rows
+            rows::slab_prep_kernel<<<static_cast<unsigned>(rws), rows::ROW_THREADS, 0, st>>>(
+                zs, plan.ldz, Hs, shape->ldH, d, y + r0, valid ? valid + r0 : nullptr, lse + r0, weight + r0, z_label + r0,
+                ref + r0, V, a_row + r0, h_scaled);
+            if (tmap_mn_major(&tmH_mn, h_scaled, rws, shape->d, shape->d) != CAT_OK) return CAT_ERR_CUDA;
+        }
         if (cudaGetLastError() != cudaSuccess) return CAT_ERR_CUDA;
         mark(st);
         {   // dH[r0 : r0 + rws, :] = (g/N) dz W : the whole vocabulary is contracted, written once
@@ -575,6 +600,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             tc::EpiOut::Params ep;
             memset(&ep, 0, sizeof(ep));
             ep.alpha = scale; ep.M = static_cast<int>(rws); ep.N = d;
+            if (!kd) ep.row_scale = a_row + r0;
             ep.out_bf16 = static_cast<__nv_bfloat16*>(dH) + r0 * shape->ldH; ep.ld_out = shape->ldH;
             const int rc = launch_tc<0, 1, tc::EpiOut>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
@@ -670,7 +696,7 @@ int cat_loss_launch_count(const cat_shape* shape, int pass) {
         if (shape->in_dtype != CAT_BF16)
             return cat_loss_launch_count(shape, 0) + cat_loss_launch_count(shape, 1);
         const FusedPlan p = plan_fused(shape);
-        return 1 + p.n_slabs * (1 + (p.warp_scan ? 1 : 2) + 1 + 2) + 1;
+        return 1 + p.n_slabs * (2 + (p.warp_scan ? 1 : 2) + 1 + 2) + 1;
     }
     return 0;
 }
@@ -714,7 +740,7 @@ int cat_loss_fwd(const cat_shape* shape, const void* H, const void* W, const int
         tc::EpiFwd::Params ep;
         ep.labels = reinterpret_cast<const long long*>(labels);
         ep.part_m = part_m; ep.part_l = part_l; ep.z_label = z_label; ep.T = T; ep.V = V;
-        ep.zs = nullptr; ep.ldz = 0; ep.part_stride = T;
+        ep.zs = nullptr; ep.ldz = 0; ep.part_stride = T; ep.ref = nullptr;
         const int rc = launch_tc<0, 0, tc::EpiFwd>(tmH, tmW, sched, ep, status, sm_count, st);
         if (rc != CAT_OK) return rc;
     } else {
@@ -900,7 +926,7 @@ int cat_loss_fwd_bwd_events(const cat_shape* shape, const void* H, const void* W
     if (!stage_events) return CAT_ERR_NULL;
     if (check_shape(shape) != CAT_OK) return CAT_ERR_SHAPE;
     if (shape->in_dtype != CAT_BF16) return CAT_ERR_DTYPE;
-    if (n_events != 5 * plan_fused(shape).n_slabs + 3) return CAT_ERR_SHAPE;
+    if (n_events != 6 * plan_fused(shape).n_slabs + 3) return CAT_ERR_SHAPE;
     for (int i = 0; i < n_events; ++i)
         if (!stage_events[i]) return CAT_ERR_NULL;
     return fused_core(shape, H, W, labels, valid, conf_ext, grad_loss, loss, lse, conf, weight, stats, dH, dW, accumulate_dW,

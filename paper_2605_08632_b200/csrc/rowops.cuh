@@ -252,50 +252,75 @@ __global__ void __launch_bounds__(1024) count_valid_kernel(const long long* labe
     }
 }
 
-// Fused path: turn one row of stored fp16 logits into bf16 dz in place,
-//   dz[r, v] = weight_r * (exp(z[r, v] - lse_r) - [v == y_r]),
-// the label entry formed from the fp32 label logit.  One CTA per row, 16-byte vectors; columns
-// at or beyond V are written as zero.  Pure streaming: 2 bytes read + 2 bytes written per logit.
-__global__ void __launch_bounds__(ROW_THREADS) z_to_dz_kernel(void* zs, long long ldz, const long long* labels,
-                                                              const unsigned char* valid, const float* lse,
-                                                              const float* weight, const float* z_label, int V) {
+// One-call path, before the logits GEMM of a row slab: the per-row reference of the stored
+// softmax numerators, ref[r] = z[r, y_r] = H[r, :] . W[y_r, :] as an fp32 dot product (one warp per
+// row).  Any finite per-row constant would do; the label logit keeps exp(z - ref) near the
+// probabilities' ratio to the label's.  Rows that take no part get 0.
+__global__ void __launch_bounds__(ROW_THREADS) label_ref_kernel(const __nv_bfloat16* H, long long ldH, const __nv_bfloat16* W,
+                                                                long long ldW, int d, const long long* labels,
+                                                                const unsigned char* valid, int n_rows, int V, float* ref) {
+    const int warp = (blockIdx.x * ROW_THREADS + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= n_rows) return;
+    const long long y = labels[warp];
+    float acc = 0.f;
+    if ((valid == nullptr || valid[warp] != 0) && y >= 0 && y < V) {
+        const uint4* h = reinterpret_cast<const uint4*>(H + static_cast<size_t>(warp) * ldH);
+        const uint4* w = reinterpret_cast<const uint4*>(W + static_cast<size_t>(y) * ldW);
+        for (int i = lane; i < d / 8; i += 32) {
+            const uint4 a = h[i], b = w[i];
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[j]));
+                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[j]));
+                acc = fmaf(fa.x, fb.x, acc);
+                acc = fmaf(fa.y, fb.y, acc);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    }
+    if (lane == 0) ref[warp] = acc;
+}
+
+// One-call path, after the row kernel of a slab (lse and weights known).  With the slab holding
+// e[r, v] = exp(z[r, v] - ref[r]), the backward's dz[r, v] = weight[r] * (exp(z - lse) - [v == y_r])
+// equals a[r] * e'[r, v], where a[r] = weight[r] * exp(ref[r] - lse[r]) and e' is e with the label
+// entry lowered by exp(lse[r] - ref[r]).  One CTA per row:
+//   * a[r] (0 for rows that take no part) for the dH GEMM's epilogue;
+//   * the label entry of the slab row patched in place (from the fp32 label logit);
+//   * Hs[r, :] = a[r] * H[r, :] in bf16, the dW GEMM's second operand (the factor rides on the
+//     contraction index there, so it has to sit in an operand).
+__global__ void __launch_bounds__(ROW_THREADS) slab_prep_kernel(void* zs, long long ldz, const __nv_bfloat16* H, long long ldH,
+                                                                int d, const long long* labels, const unsigned char* valid,
+                                                                const float* lse, const float* weight, const float* z_label,
+                                                                const float* ref, int V, float* a_out, __nv_bfloat16* Hs) {
     const int r = blockIdx.x;
     const long long y = labels[r];
     const bool ok = (valid == nullptr || valid[r] != 0) && y >= 0 && y < V;
-    const float w = ok ? weight[r] : 0.f;
-    const float l2 = ok ? lse[r] * 1.4426950408889634f : INFINITY;
-    const int yi = ok ? static_cast<int>(y) : -1;
-    const float dz_label = ok ? w * (expf(z_label[r] - lse[r]) - 1.f) : 0.f;
-    uint4* row = reinterpret_cast<uint4*>(static_cast<unsigned short*>(zs) + static_cast<size_t>(r) * ldz);
-    const int groups = static_cast<int>(ldz / 8);
-    for (int gi = threadIdx.x; gi < groups; gi += ROW_THREADS) {
-        const uint4 in = __ldcs(row + gi);
+    const float a = ok ? weight[r] * expf(ref[r] - lse[r]) : 0.f;
+    if (threadIdx.x == 0) {
+        a_out[r] = a;
+        if (ok) {
+            // exp(lse - ref) = 1 / (probability of the label) when ref is the label logit; capped like the slab
+            const float e_label = expf(fminf(z_label[r] - ref[r], 79.f)) - expf(fminf(lse[r] - ref[r], 79.f));
+            reinterpret_cast<__nv_bfloat16*>(zs)[static_cast<size_t>(r) * ldz + y] = __float2bfloat16_rn(e_label);
+        }
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(H + static_cast<size_t>(r) * ldH);
+    uint4* dst = reinterpret_cast<uint4*>(Hs + static_cast<size_t>(r) * d);
+    for (int i = threadIdx.x; i < d / 8; i += ROW_THREADS) {
+        const uint4 in = src[i];
         const uint32_t wds[4] = {in.x, in.y, in.z, in.w};
-        float f[8];
+        uint32_t o[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&wds[i]));
-            f[2 * i] = t.x;
-            f[2 * i + 1] = t.y;
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[j]));
+            __nv_bfloat162 b = __floats2bfloat162_rn(a * f.x, a * f.y);
+            o[j] = *reinterpret_cast<uint32_t*>(&b);
         }
-        const int col = gi * 8;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float pz;
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pz) : "f"(fmaf(f[i], 1.4426950408889634f, -l2)));
-            f[i] = (col + i < V) ? w * pz : 0.f;
-            if (col + i == yi) f[i] = dz_label;
-        }
-        uint4 out;
-        __nv_bfloat162 b0 = __floats2bfloat162_rn(f[0], f[1]);
-        __nv_bfloat162 b1 = __floats2bfloat162_rn(f[2], f[3]);
-        __nv_bfloat162 b2 = __floats2bfloat162_rn(f[4], f[5]);
-        __nv_bfloat162 b3 = __floats2bfloat162_rn(f[6], f[7]);
-        out.x = *reinterpret_cast<uint32_t*>(&b0);
-        out.y = *reinterpret_cast<uint32_t*>(&b1);
-        out.z = *reinterpret_cast<uint32_t*>(&b2);
-        out.w = *reinterpret_cast<uint32_t*>(&b3);
-        row[gi] = out;
+        dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 

@@ -101,16 +101,24 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
 
 // Forward: online max / sum-exp over the vocabulary (softmax partition function of Eq. 11's
 // log P), and the label logit z[r, y_r] picked from the accumulator chunk that holds it.
-// STORE = true additionally writes the logits of the tile as fp16 (saturating) into a row slab,
-// for the fused forward+backward path that keeps one slab of logits instead of recomputing them.
-template <bool STORE>
+// STORE = 1 additionally writes the logits of the tile as fp16 (saturating) into a row slab
+// (the distillation path, which needs the logits of both models side by side).
+// STORE = 2 writes e[r, v] = exp(z[r, v] - ref[r]) as bf16 instead: softmax numerators relative to
+// a per-row reference fixed before the GEMM (the row's label logit), so that later
+// softmax[r, v] = exp(ref[r] - lse[r]) * e[r, v] needs only a per-row factor, which the dH / dW
+// GEMMs absorb, and no second pass over the slab.  The exponent is capped at EXP_CAP_LOG2 so that
+// e stays finite whatever the inputs.
+constexpr float EXP_CAP_LOG2 = 115.0f;   // 2^115 = e^79.7
+
+template <int STORE>
 struct EpiFwdT {
     struct Params {
         const long long* labels;   // [T]
         float* part_m;             // [n_groups][part_stride] running max of each (row, vocabulary split)
         float* part_l;             // [n_groups][part_stride] sum exp(z - max)
         float* z_label;            // [T]
-        __half* zs;                // [T][ldz] fp16 logits (STORE only)
+        __half* zs;                // [T][ldz] 16-bit slab: fp16 logits (STORE 1) or bf16 exp(z - ref) (STORE 2)
+        const float* ref;          // [T] per-row reference (STORE 2 only)
         long long ldz;
         long long part_stride;
         int T;
@@ -118,6 +126,7 @@ struct EpiFwdT {
     };
     struct State {
         float m_run, l_run;
+        float ref2;                // ref[row] * log2(e)
         int y;
         int row;
     };
@@ -125,10 +134,12 @@ struct EpiFwdT {
         s.row = m_tile * BM + row_in_tile;
         s.m_run = -INFINITY;
         s.l_run = 0.f;
+        s.ref2 = 0.f;
         s.y = -1;
         if (s.row < p.T) {
             const long long y = p.labels[s.row];
             if (y >= 0 && y < p.V) s.y = static_cast<int>(y);
+            if (STORE == 2) s.ref2 = p.ref[s.row] * LOG2E;
         }
     }
     __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
@@ -149,7 +160,25 @@ struct EpiFwdT {
                 for (int i = 0; i < 32; ++i)
                     if (i >= live) f[i] = -INFINITY;
             }
-            if (STORE) {
+            if (STORE == 2) {
+                if (s.row < p.T) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float e[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            e[i] = ptx::ex2_approx(fminf(fmaf(f[q * 8 + i], LOG2E, -s.ref2), EXP_CAP_LOG2));
+                        uint4 pk;
+                        pk.x = ptx::pack_bf16x2(e[0], e[1]);
+                        pk.y = ptx::pack_bf16x2(e[2], e[3]);
+                        pk.z = ptx::pack_bf16x2(e[4], e[5]);
+                        pk.w = ptx::pack_bf16x2(e[6], e[7]);
+                        __stcs(dst + q, pk);
+                    }
+                }
+            }
+            if (STORE == 1) {
                 if (s.row < p.T) {
                     uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
 #pragma unroll
@@ -190,8 +219,9 @@ struct EpiFwdT {
         }
     }
 };
-using EpiFwd = EpiFwdT<false>;
-using EpiFwdStore = EpiFwdT<true>;
+using EpiFwd = EpiFwdT<0>;
+using EpiFwdStore = EpiFwdT<1>;
+using EpiFwdExp = EpiFwdT<2>;
 
 // Backward recompute: dz[r, v] = weight_r * (exp(z - lse_r) - [v == y_r]) as a bf16 tile of the
 // current vocabulary slab (the scalar g/N is applied later, in fp32, by the dH / dW epilogues).
@@ -275,6 +305,7 @@ struct EpiDz {
 struct EpiOut {
     struct Params {
         const float* alpha;            // device scalar or nullptr (= 1)
+        const float* row_scale;        // [M] per-output-row factor or nullptr (= 1)
         const float* add_f32;          // [M][ld_add] or nullptr
         const __nv_bfloat16* add_bf16; // [M][ld_add] or nullptr
         float* out_f32;                // [M][ld_out] or nullptr
@@ -289,6 +320,7 @@ struct EpiOut {
     __device__ static __forceinline__ void begin_item(const Params& p, State& s, int m_tile, int row_in_tile) {
         s.row = m_tile * BM + row_in_tile;
         s.alpha = p.alpha ? *p.alpha : 1.f;
+        if (p.row_scale && s.row < p.M) s.alpha *= p.row_scale[s.row];
     }
     __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
         const int col0 = n_tile * BN;

@@ -58,7 +58,7 @@ def test_workspace_sizes():
     assert fwd <= conf_ws < 2 * fwd + (1 << 20) and B.cat_loss_workspace_bytes(s, 4) == 0
     assert B.cat_loss_launch_count(s, 3) == 3
     assert B.cat_loss_launch_count(s, 0) == 3 and B.cat_loss_launch_count(s, 1) == 7
-    assert B.cat_loss_launch_count(s, 2) == 1 + 2 * 5 + 1
+    assert B.cat_loss_launch_count(s, 2) == 1 + 2 * 6 + 1
 
 
 @pytest.mark.parametrize("kw,code", [
