@@ -35,6 +35,9 @@ import torch
 # first row slab of the one-call path, ncu_two_call_gemms_config2.md for the two-call forward).
 # Valid for that kernel, workload and T only; None for anything else.
 TRAFFIC_BYTES = {
+    ("config2", 16384, "logits"): 684621000 + 2392343000,
+    ("config2", 16384, "dH"): 5998683000 + 34431000,
+    ("config2", 16384, "dW"): 5164804000 + 1037821000,
     ("config2", 16384, "fwd_two_call"): 2848929024 + 21131008,
 }
 STAGES = ("label_ref", "logits", "rows", "slab_prep", "dH", "dW")

@@ -192,6 +192,32 @@ def test_fused_call_with_stage_events_gives_the_same_bits_and_ordered_times():
                                   cl.lse, cl.conf, cl.weight, cl.stats, cl.dH, cl.dW, False, cl._ws_fused, evs[:-1])
 
 
+def test_one_call_path_with_a_label_far_below_the_row_maximum():
+    # The one-call path keeps exp(z - label logit) with the exponent capped at 79.7.  Give one row a logit
+    # ~120 above its label's: everything stays finite, loss / lse / confidence are exact, every other
+    # row's gradient is untouched, and that row's own gradient is damped, never amplified.  The two-call
+    # path has no cap and matches the oracle on the whole batch.
+    batch = synth.make_batch(2, T=256, d=128, V=1000)
+    r, v_star = 8, 123                                              # position 0 of block 1: weight 1
+    assert int(batch.labels[r]) != v_star
+    Wv = batch.W[v_star].double()
+    batch.H[r] = (120.0 * Wv / (Wv * Wv).sum()).to(batch.H.dtype)
+    fwd, dH, dW = run_oracle(batch)
+    assert fwd["row_ce"][r] > 85.0
+    two = run_gpu(batch)
+    check_forward(two, fwd, batch.K, batch.torch_dtype, batch.V)
+    check_backward(two, fwd, dH, dW, batch.K, batch.torch_dtype, per_position=False)
+    one = run_gpu_fused(batch)
+    check_forward(one, fwd, batch.K, batch.torch_dtype, batch.V)
+    assert np.isfinite(one["dH"]).all() and np.isfinite(one["dW"]).all()
+    others = np.setdiff1d(np.arange(batch.T), [r])
+    assert rel_l2(one["dH"][others], dH[others]) <= 1e-2
+    n_gpu, n_ref = np.linalg.norm(one["dH"][r]), np.linalg.norm(dH[r])
+    assert 0.0 < n_gpu <= 1.01 * n_ref
+    cos = float(one["dH"][r] @ dH[r]) / (n_gpu * n_ref)
+    assert cos > 0.99                                               # same direction
+
+
 def test_errors_on_gpu_box_leave_context_usable():
     s = B.make_shape(64, 128, 512, 8, B.CAT_BF16)
     x = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
