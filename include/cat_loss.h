@@ -201,8 +201,10 @@ int cat_count_valid(const cat_shape* shape, const int64_t* labels, const uint8_t
  * exceeds one slab unit, so a T x V matrix never exists at once) and bf16 rounding of the stored
  * numerators (relative 2^-9, the same as rounding dz to bf16).  The exponent z - ref is capped at
  * 79.7 so that e stays finite for any input: only a row whose label is more than 79.7 nats below
- * the row's largest logit (label probability under 1e-34) gets a damped gradient; its loss, lse and
- * confidence are exact.
+ * the row's largest logit (label probability under 1e-34) gets a damped gradient, and none at all
+ * once exp(ref - lse) underflows binary32 (label probability under about 1e-45, where the fp32
+ * confidence is zero as well); its loss and lse are exact.  cat_loss_fwd + cat_loss_bwd have no such
+ * limit.
  * Arguments as in cat_loss_fwd and cat_loss_bwd; workspace of
  * cat_loss_workspace_bytes(shape, 2) bytes; cat_loss_launch_count(shape, 2) kernels.
  * For CAT_F32 inputs this runs the fp32 forward and backward passes back to back.

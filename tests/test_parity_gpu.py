@@ -194,9 +194,10 @@ def test_fused_call_with_stage_events_gives_the_same_bits_and_ordered_times():
 
 def test_one_call_path_with_a_label_far_below_the_row_maximum():
     # The one-call path keeps exp(z - label logit) with the exponent capped at 79.7.  Give one row a logit
-    # ~120 above its label's: everything stays finite, loss / lse / confidence are exact, every other
-    # row's gradient is untouched, and that row's own gradient is damped, never amplified.  The two-call
-    # path has no cap and matches the oracle on the whole batch.
+    # ~120 above its label's (label probability e^-120, below what binary32 holds): everything stays
+    # finite, loss / lse / confidence are exact, every other row's gradient is untouched, and that row's
+    # own gradient is damped (here to zero, its factor exp(ref - lse) underflows), never amplified.
+    # The two-call path has no cap and matches the oracle on the whole batch.
     batch = synth.make_batch(2, T=256, d=128, V=1000)
     r, v_star = 8, 123                                              # position 0 of block 1: weight 1
     assert int(batch.labels[r]) != v_star
@@ -213,9 +214,9 @@ def test_one_call_path_with_a_label_far_below_the_row_maximum():
     others = np.setdiff1d(np.arange(batch.T), [r])
     assert rel_l2(one["dH"][others], dH[others]) <= 1e-2
     n_gpu, n_ref = np.linalg.norm(one["dH"][r]), np.linalg.norm(dH[r])
-    assert 0.0 < n_gpu <= 1.01 * n_ref
-    cos = float(one["dH"][r] @ dH[r]) / (n_gpu * n_ref)
-    assert cos > 0.99                                               # same direction
+    assert n_gpu <= 1.01 * n_ref
+    if n_gpu > 0:
+        assert float(one["dH"][r] @ dH[r]) / (n_gpu * n_ref) > 0.99   # same direction
 
 
 def test_errors_on_gpu_box_leave_context_usable():
