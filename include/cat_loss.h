@@ -261,7 +261,7 @@ int cat_loss_fused_slabs(const cat_shape* shape, int64_t* row_begin, int capacit
  *   - Arguments are those of cat_loss_fwd without `workspace` / `workspace_bytes`.
  *   - Shapes whose cat_loss_workspace_bytes(shape, 0) exceeds CAT_STATIC_SCRATCH_BYTES are
  *     refused with CAT_ERR_LIMIT before anything is launched (config 2, T=16384 x V=128256,
- *     needs 16.7 MB and fits; T=32768 with 128 vocabulary splits does not).
+ *     needs 16.7 MB and fits; T=65536 rows of the same head need 33.6 MB and do not).
  *   - The first call on each device looks up the array's device address (once per device,
  *     with that device current).  Make that first call outside any stream capture.
  *   - All calls share the one array and it keeps whatever the last call left in it; the
