@@ -524,7 +524,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
             constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM * CG, BN, A_MN, B_MN);
+            // The tensor pipe takes only a few MMAs ahead of the one it executes, so the instructions between
+            // two issues are on its critical path: the shared-memory descriptors of stage 0 are built once and
+            // those of the other stages and k-slices follow by adding to the (address >> 4) field.
+            //   K-major: 16 elements = 32 bytes further inside the 128-byte swizzle row;
+            //   MN-major: 16 k-rows = two 8-row swizzle atoms (2048 bytes) further.
+            const uint64_t adesc0 = A_MN ? ptx::smem_desc_sw128(ring, MN_ATOM_BYTES, 1024) : ptx::smem_desc_sw128(ring, 16, 1024);
+            const uint64_t bdesc0 = B_MN ? ptx::smem_desc_sw128(ring + A_STAGE_BYTES, MN_ATOM_BYTES, 1024)
+                                         : ptx::smem_desc_sw128(ring + A_STAGE_BYTES, 16, 1024);
+            constexpr uint64_t STAGE_STEP = G::STAGE_BYTES >> 4;
+            constexpr uint64_t A_KSTEP = (A_MN ? 2048 : 32) >> 4;
+            constexpr uint64_t B_KSTEP = (B_MN ? 2048 : 32) >> 4;
+            const uint32_t full0 = ptx::smem_u32(&ctl.full[0]), empty0 = ptx::smem_u32(&ctl.empty[0]);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            uint64_t adesc = adesc0, bdesc = bdesc0;
             bool ok = true;
             for (int item = worker; item < sched.n_items && ok; item += n_workers) {
                 int m_tile, group, n_begin, n_end;
@@ -534,25 +547,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem + acc * BN;
                     for (int kb = 0; kb < sched.num_kb; ++kb) {
-                        if (!wait_bounded(ptx::smem_u32(&ctl.full[stage]), phase, abort, status)) { ok = false; break; }
+                        if (!wait_bounded(full0 + stage * 8u, phase, abort, status)) { ok = false; break; }
                         ptx::tc_fence_after();
-                        const uint32_t a_base = ring + stage * G::STAGE_BYTES;
-                        const uint32_t b_base = a_base + A_STAGE_BYTES;
 #pragma unroll
                         for (int j = 0; j < BK / 16; ++j) {
-                            // K-major: 16 elements = 32 bytes further inside the 128-byte swizzle row.
-                            // MN-major: 16 k-rows = two 8-row swizzle atoms (2048 bytes) further.
-                            const uint64_t adesc = A_MN ? ptx::smem_desc_sw128(a_base + j * 2048, MN_ATOM_BYTES, 1024)
-                                                        : ptx::smem_desc_sw128(a_base + j * 32, 16, 1024);
-                            const uint64_t bdesc = B_MN ? ptx::smem_desc_sw128(b_base + j * 2048, MN_ATOM_BYTES, 1024)
-                                                        : ptx::smem_desc_sw128(b_base + j * 32, 16, 1024);
-                            if (CG == 1) ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
-                            else ptx::umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
+                            const uint32_t accumulate = (j != 0 || kb != 0) ? 1u : 0u;
+                            if (CG == 1) ptx::umma_bf16(d_tmem, adesc + j * A_KSTEP, bdesc + j * B_KSTEP, idesc, accumulate);
+                            else ptx::umma_bf16_pair(d_tmem, adesc + j * A_KSTEP, bdesc + j * B_KSTEP, idesc, accumulate);
                         }
                         // frees the stage (in both CTAs of a pair) once these MMAs have read it
-                        if (CG == 1) ptx::umma_commit(ptx::smem_u32(&ctl.empty[stage]));
-                        else ptx::umma_commit_pair(ptx::smem_u32(&ctl.empty[stage]), 3);
-                        if (++stage == G::STAGES) { stage = 0; phase ^= 1u; }
+                        if (CG == 1) ptx::umma_commit(empty0 + stage * 8u);
+                        else ptx::umma_commit_pair(empty0 + stage * 8u, 3);
+                        if (++stage == G::STAGES) {
+                            stage = 0; phase ^= 1u; adesc = adesc0; bdesc = bdesc0;
+                        } else {
+                            adesc += STAGE_STEP; bdesc += STAGE_STEP;
+                        }
                     }
                     if (!ok) break;
                     // accumulator complete (in both CTAs of a pair)
