@@ -199,8 +199,9 @@ int cat_count_valid(const cat_shape* shape, const int64_t* labels, const uint8_t
  * 6*T*d*V flops of the three contractions instead of 8*T*d*V; the price is one slab of 16-bit values
  * in the workspace (at most about slab_mib MiB, default 2560, and always at least two slabs once T
  * exceeds one slab unit, so a T x V matrix never exists at once) and bf16 rounding of the stored
- * numerators (relative 2^-9, the same as rounding dz to bf16).  The exponent z - ref is capped at
- * 79.7 so that e stays finite for any input: only a row whose label is more than 79.7 nats below
+ * numerators (relative 2^-9, the same as rounding dz to bf16).  e is formed as exp(z - m) * exp(m - ref),
+ * m the running row maximum, with m - ref capped at 79.7 so that e stays finite for any input: only a
+ * row whose label is more than 79.7 nats below
  * the row's largest logit (label probability under 1e-34) gets a damped gradient, and none at all
  * once exp(ref - lse) underflows binary32 (label probability under about 1e-45, where the fp32
  * confidence is zero as well); its loss and lse are exact.  cat_loss_fwd + cat_loss_bwd have no such

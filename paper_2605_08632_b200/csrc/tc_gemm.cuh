@@ -106,8 +106,9 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
 // STORE = 2 writes e[r, v] = exp(z[r, v] - ref[r]) as bf16 instead: softmax numerators relative to
 // a per-row reference fixed before the GEMM (the row's label logit), so that later
 // softmax[r, v] = exp(ref[r] - lse[r]) * e[r, v] needs only a per-row factor, which the dH / dW
-// GEMMs absorb, and no second pass over the slab.  The exponent is capped at EXP_CAP_LOG2 so that
-// e stays finite whatever the inputs.
+// GEMMs absorb, and no second pass over the slab.  e is formed as exp(z - m) * exp(m - ref) with m the
+// running maximum, the second factor's exponent capped at EXP_CAP_LOG2, so e stays finite whatever
+// the inputs.
 constexpr float EXP_CAP_LOG2 = 115.0f;   // 2^115 = e^79.7
 
 template <int STORE>
@@ -160,24 +161,6 @@ struct EpiFwdT {
                 for (int i = 0; i < 32; ++i)
                     if (i >= live) f[i] = -INFINITY;
             }
-            if (STORE == 2) {
-                if (s.row < p.T) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float e[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            e[i] = ptx::ex2_approx(fminf(fmaf(f[q * 8 + i], LOG2E, -s.ref2), EXP_CAP_LOG2));
-                        uint4 pk;
-                        pk.x = ptx::pack_bf16x2(e[0], e[1]);
-                        pk.y = ptx::pack_bf16x2(e[2], e[3]);
-                        pk.z = ptx::pack_bf16x2(e[4], e[5]);
-                        pk.w = ptx::pack_bf16x2(e[6], e[7]);
-                        __stcs(dst + q, pk);
-                    }
-                }
-            }
             if (STORE == 1) {
                 if (s.row < p.T) {
                     uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
@@ -200,14 +183,54 @@ struct EpiFwdT {
                     if (i == rel) zy = f[i];
                 p.z_label[s.row] = zy;
             }
-            float cmax = f[0];
+            float cmax = ptx::max3_f32(f[0], f[1], f[2]);
 #pragma unroll
-            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, f[i]);
+            for (int i = 3; i + 1 < 32; i += 2) cmax = ptx::max3_f32(cmax, f[i], f[i + 1]);
+            cmax = fmaxf(cmax, f[31]);
             const float m_new = fmaxf(s.m_run, cmax);
             const float mb = m_new * LOG2E;
             float sum = 0.f;
+            if (STORE == 2) {
+                // One exponential per logit serves both uses: exp(z - m) for the running sum, and
+                // exp(z - ref) = exp(z - m) * exp(m - ref) for the slab (the factor capped so that the product
+                // stays finite).  The scale, sum and product run on packed fp32 pairs.
+                const uint64_t l2e2 = ptx::pack_f32x2(LOG2E, LOG2E), nmb2 = ptx::pack_f32x2(-mb, -mb);
+                const float fac = ptx::ex2_approx(fminf(mb - s.ref2, EXP_CAP_LOG2));
+                const uint64_t fac2 = ptx::pack_f32x2(fac, fac);
+                uint64_t sum2 = ptx::pack_f32x2(0.f, 0.f);
+                uint32_t packed[16];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) sum += ptx::ex2_approx(fmaf(f[i], LOG2E, -mb));
+                for (int i = 0; i < 16; ++i) {
+                    float x0, x1;
+                    ptx::unpack_f32x2(ptx::fma_f32x2(ptx::pack_f32x2(f[2 * i], f[2 * i + 1]), l2e2, nmb2), x0, x1);
+                    const uint64_t e2 = ptx::pack_f32x2(ptx::ex2_approx(x0), ptx::ex2_approx(x1));
+                    sum2 = ptx::add_f32x2(sum2, e2);
+                    float y0, y1;
+                    ptx::unpack_f32x2(ptx::mul_f32x2(e2, fac2), y0, y1);
+                    packed[i] = ptx::pack_bf16x2(y0, y1);
+                }
+                float s0, s1;
+                ptx::unpack_f32x2(sum2, s0, s1);
+                sum = s0 + s1;
+                if (s.row < p.T) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        __stcs(dst + q, make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]));
+                }
+            } else {
+                const uint64_t l2e2 = ptx::pack_f32x2(LOG2E, LOG2E), nmb2 = ptx::pack_f32x2(-mb, -mb);
+                uint64_t sum2 = ptx::pack_f32x2(0.f, 0.f);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float x0, x1;
+                    ptx::unpack_f32x2(ptx::fma_f32x2(ptx::pack_f32x2(f[2 * i], f[2 * i + 1]), l2e2, nmb2), x0, x1);
+                    sum2 = ptx::add_f32x2(sum2, ptx::pack_f32x2(ptx::ex2_approx(x0), ptx::ex2_approx(x1)));
+                }
+                float s0, s1;
+                ptx::unpack_f32x2(sum2, s0, s1);
+                sum = s0 + s1;
+            }
             s.l_run = fmaf(s.l_run, ptx::ex2_approx((s.m_run - m_new) * LOG2E), sum);
             s.m_run = m_new;
         }
