@@ -386,7 +386,7 @@ tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int b
     tc::Sched s;
     s.num_m_tiles = static_cast<int>(cdiv(M, tile_m()));
     s.num_n_tiles = static_cast<int>(cdiv(N, tc::BN));
-    s.num_kb = static_cast<int>(cdiv(Kd, tc::BK));
+    s.num_kb = static_cast<int>(cdiv(Kd, tc::BK * (cta_group() == 2 ? tc::Geo<2>::KS : tc::Geo<1>::KS)));   // ring stages along the contraction
     s.n_groups = n_groups > 0 ? n_groups : s.num_n_tiles;
     s.band_m = band_m < 1 ? 1 : band_m;
     s.n_fastest = n_fastest;

@@ -39,7 +39,7 @@ constexpr float LOG2E = 1.4426950408889634f;
 struct Sched {
     int num_m_tiles;   // tiles of BM rows of the output
     int num_n_tiles;   // tiles of BN columns of the output
-    int num_kb;        // blocks of BK along the contraction
+    int num_kb;        // ring stages (BK * k-slices per stage) along the contraction
     int n_groups;      // column groups per m-tile: one item = (m-tile, group); a group is a run of n-tiles
     int band_m;        // m-tiles per band when m runs fastest (keeps a band of A rows L2-resident)
     int n_fastest;     // 1: items ordered group-fastest within an m-tile; 0: m-fastest within (band, group)
@@ -291,10 +291,19 @@ struct EpiDz {
             ptx::tmem_ld_wait();
             float f[32];
             const int live = ncols - c * 32;
+            {   // w * exp2(z * log2e - lse * log2e) on packed fp32 pairs
+                const uint64_t l2e2 = ptx::pack_f32x2(LOG2E, LOG2E), nl2 = ptx::pack_f32x2(-s.l2, -s.l2), w2 = ptx::pack_f32x2(s.w, s.w);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float pz = ptx::ex2_approx(fmaf(__uint_as_float(v[i]), LOG2E, -s.l2));
-                f[i] = (i < live) ? s.w * pz : 0.f;
+                for (int i = 0; i < 16; ++i) {
+                    float x0, x1;
+                    ptx::unpack_f32x2(ptx::fma_f32x2(ptx::pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), l2e2, nl2), x0, x1);
+                    ptx::unpack_f32x2(ptx::mul_f32x2(ptx::pack_f32x2(ptx::ex2_approx(x0), ptx::ex2_approx(x1)), w2), f[2 * i], f[2 * i + 1]);
+                }
+            }
+            if (live < 32) {   // ragged last tile of the vocabulary
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i >= live) f[i] = 0.f;
             }
             const int rel = s.y_rel - (col0 + c * 32);
             if (rel >= 0 && rel < 32) {
@@ -417,12 +426,24 @@ struct EpiOut {
 //   `tfull` are signalled in both CTAs at once by the leader's tcgen05.commit; `tempty` lives in
 //   the leader and collects one arrival per epilogue warp of both CTAs.
 // ------------------------------------------------------------------------------------------
+// one TMA box; in pair mode the byte count may be signalled on the peer's barrier
+template <int CG>
+__device__ __forceinline__ void load_box(uint32_t dst, const CUtensorMap* m, int x, int y, uint32_t bar) {
+    if (CG == 1) ptx::tma_load_2d(dst, m, x, y, bar);
+    else ptx::tma_load_2d_pair(dst, m, x, y, bar);
+}
+
+constexpr int PAIR_KSLICES = 2;   // BK-wide k-slices per ring stage in pair mode (1: six 32 KB stages, 2: three 64 KB stages)
+
 template <int CG>
 struct Geo {
-    static constexpr int STAGES = CG == 1 ? 4 : 6;
+    static constexpr int KS = CG == 1 ? 1 : PAIR_KSLICES;        // k-slices of BK per stage
+    static constexpr int STAGES = CG == 1 ? 4 : 6 / KS;
     static constexpr int BN_CTA = BN / CG;                        // B-tile rows this CTA loads
-    static constexpr int B_BYTES = BN_CTA * BK * 2;
-    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_BYTES;
+    static constexpr int B_SLICE_BYTES = BN_CTA * BK * 2;
+    static constexpr int A_BYTES = A_STAGE_BYTES * KS;
+    static constexpr int B_BYTES = B_SLICE_BYTES * KS;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
     static constexpr int TILE_M = BM * CG;                        // output rows per scheduled m-tile
 };
@@ -488,38 +509,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         if (!wait_bounded(ptx::smem_u32(&ctl.empty[stage]), phase ^ 1u, abort, status)) { ok = false; break; }
                         const uint32_t full_local = ptx::smem_u32(&ctl.full[stage]);
                         if (leader) ptx::mbar_arrive_expect_tx(full_local, G::STAGE_BYTES * CG);
-                        const uint32_t a_dst = ring + stage * G::STAGE_BYTES;
-                        const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                        if (CG == 1) {
+                        const uint32_t full_sig = CG == 1 ? full_local : ptx::mapa_shared(full_local, 0);   // pair: the leader's barrier
+#pragma unroll
+                        for (int h = 0; h < G::KS; ++h) {
+                            const uint32_t a_dst = ring + stage * G::STAGE_BYTES + h * A_STAGE_BYTES;
+                            const uint32_t b_dst = ring + stage * G::STAGE_BYTES + G::A_BYTES + h * G::B_SLICE_BYTES;
+                            const int k0 = (kb * G::KS + h) * BK;
                             if (A_MN) {
 #pragma unroll
-                                for (int j = 0; j < BM / 64; ++j)
-                                    ptx::tma_load_2d(a_dst + j * MN_ATOM_BYTES, &tmA, m0 + j * 64, kb * BK, full_local);
+                                for (int j = 0; j < BM / 64; ++j) load_box<CG>(a_dst + j * MN_ATOM_BYTES, &tmA, m0 + j * 64, k0, full_sig);
                             } else {
-                                ptx::tma_load_2d(a_dst, &tmA, kb * BK, m0, full_local);
+                                load_box<CG>(a_dst, &tmA, k0, m0, full_sig);
                             }
                             if (B_MN) {
 #pragma unroll
-                                for (int j = 0; j < G::BN_CTA / 64; ++j)
-                                    ptx::tma_load_2d(b_dst + j * MN_ATOM_BYTES, &tmB, n0 + j * 64, kb * BK, full_local);
+                                for (int j = 0; j < G::BN_CTA / 64; ++j) load_box<CG>(b_dst + j * MN_ATOM_BYTES, &tmB, n0 + j * 64, k0, full_sig);
                             } else {
-                                ptx::tma_load_2d(b_dst, &tmB, kb * BK, n0, full_local);
-                            }
-                        } else {
-                            const uint32_t full_lead = ptx::mapa_shared(full_local, 0);   // the leader's barrier
-                            if (A_MN) {
-#pragma unroll
-                                for (int j = 0; j < BM / 64; ++j)
-                                    ptx::tma_load_2d_pair(a_dst + j * MN_ATOM_BYTES, &tmA, m0 + j * 64, kb * BK, full_lead);
-                            } else {
-                                ptx::tma_load_2d_pair(a_dst, &tmA, kb * BK, m0, full_lead);
-                            }
-                            if (B_MN) {
-#pragma unroll
-                                for (int j = 0; j < G::BN_CTA / 64; ++j)
-                                    ptx::tma_load_2d_pair(b_dst + j * MN_ATOM_BYTES, &tmB, n0 + j * 64, kb * BK, full_lead);
-                            } else {
-                                ptx::tma_load_2d_pair(b_dst, &tmB, kb * BK, n0, full_lead);
+                                load_box<CG>(b_dst, &tmB, k0, n0, full_sig);
                             }
                         }
                         ++issued;
@@ -553,8 +559,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             //   K-major: 16 elements = 32 bytes further inside the 128-byte swizzle row;
             //   MN-major: 16 k-rows = two 8-row swizzle atoms (2048 bytes) further.
             const uint64_t adesc0 = A_MN ? ptx::smem_desc_sw128(ring, MN_ATOM_BYTES, 1024) : ptx::smem_desc_sw128(ring, 16, 1024);
-            const uint64_t bdesc0 = B_MN ? ptx::smem_desc_sw128(ring + A_STAGE_BYTES, MN_ATOM_BYTES, 1024)
-                                         : ptx::smem_desc_sw128(ring + A_STAGE_BYTES, 16, 1024);
+            const uint64_t bdesc0 = B_MN ? ptx::smem_desc_sw128(ring + G::A_BYTES, MN_ATOM_BYTES, 1024)
+                                         : ptx::smem_desc_sw128(ring + G::A_BYTES, 16, 1024);
+            constexpr uint64_t A_SLICE_STEP = A_STAGE_BYTES >> 4, B_SLICE_STEP = G::B_SLICE_BYTES >> 4;
             constexpr uint64_t STAGE_STEP = G::STAGE_BYTES >> 4;
             constexpr uint64_t A_KSTEP = (A_MN ? 2048 : 32) >> 4;
             constexpr uint64_t B_KSTEP = (B_MN ? 2048 : 32) >> 4;
@@ -573,10 +580,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         if (!wait_bounded(full0 + stage * 8u, phase, abort, status)) { ok = false; break; }
                         ptx::tc_fence_after();
 #pragma unroll
-                        for (int j = 0; j < BK / 16; ++j) {
-                            const uint32_t accumulate = (j != 0 || kb != 0) ? 1u : 0u;
-                            if (CG == 1) ptx::umma_bf16(d_tmem, adesc + j * A_KSTEP, bdesc + j * B_KSTEP, idesc, accumulate);
-                            else ptx::umma_bf16_pair(d_tmem, adesc + j * A_KSTEP, bdesc + j * B_KSTEP, idesc, accumulate);
+                        for (int h = 0; h < G::KS; ++h) {
+#pragma unroll
+                            for (int j = 0; j < BK / 16; ++j) {
+                                const uint32_t accumulate = (h != 0 || j != 0 || kb != 0) ? 1u : 0u;
+                                const uint64_t ad = adesc + h * A_SLICE_STEP + j * A_KSTEP, bd = bdesc + h * B_SLICE_STEP + j * B_KSTEP;
+                                if (CG == 1) ptx::umma_bf16(d_tmem, ad, bd, idesc, accumulate);
+                                else ptx::umma_bf16_pair(d_tmem, ad, bd, idesc, accumulate);
+                            }
                         }
                         // frees the stage (in both CTAs of a pair) once these MMAs have read it
                         if (CG == 1) ptx::umma_commit(empty0 + stage * 8u);
