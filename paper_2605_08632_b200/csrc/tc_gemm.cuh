@@ -419,8 +419,10 @@ struct EpiOut {
 // CG = 1: one CTA per 128 x 256 output tile.
 // CG = 2: a cluster of two CTAs shares a 256 x 256 output tile (tcgen05 cta_group::2).  CTA
 //   `rank` of the pair loads the A rows of its own 128-row half and half of the B tile (128 of
-//   the 256 columns), so a stage is 32 KB instead of 48 KB per CTA and the ring holds six
-//   stages.  The leader (rank 0) issues every MMA; each CTA's accumulator half (its 128 rows x
+//   the 256 columns): 32 KB per 64-wide k-slice instead of 48 KB per CTA.  A ring stage holds
+//   two k-slices (64 KB, three stages): the MMA-issuing thread then pays the per-stage
+//   bookkeeping (commit, barrier wait, fence), which sits on the tensor pipe's critical path,
+//   once per eight MMAs instead of four.  The leader (rank 0) issues every MMA; each CTA's accumulator half (its 128 rows x
 //   256 columns) lives in its own TMEM and is drained by its own epilogue warps.  Barrier
 //   wiring: `full` lives in the leader and counts the bytes of both CTAs' loads; `empty` and
 //   `tfull` are signalled in both CTAs at once by the leader's tcgen05.commit; `tempty` lives in
