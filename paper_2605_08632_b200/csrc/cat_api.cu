@@ -339,14 +339,19 @@ inline int tmap_b(CUtensorMap* m, const void* base, long long mn, long long k, l
     return tmap_k_major(m, base, mn, k, ld, tc::BN / cta_group());
 }
 
+// Output slab [rows][cols] of 16-bit values, written by the epilogue warps as boxes of 32 rows x 64 columns.
+inline int tmap_out(CUtensorMap* m, const void* base, long long rows, long long cols, long long ld) {
+    return make_tmap(m, base, rows, cols, ld, 64, 32);
+}
+
 int band_tiles(long long d) {
     long long b = (64ll << 20) / (tile_m() * d * 2);
     return static_cast<int>(b < 1 ? 1 : b);
 }
 
 template <int A_MN, int B_MN, class Epi, int CG>
-int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& sched, const typename Epi::Params& ep,
-                 int* status, int sm_count, cudaStream_t st) {
+int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const tc::Sched& sched,
+                 const typename Epi::Params& ep, int* status, int sm_count, cudaStream_t st) {
     auto kern = tc::gemm_kernel<A_MN, B_MN, Epi, CG>;
     constexpr int smem = tc::Geo<CG>::SMEM_BYTES;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -368,18 +373,21 @@ int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tmA, tmB, sched, ep, status) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmOut, sched, ep, status) != cudaSuccess) {
         cudaGetLastError();
         return CAT_ERR_CUDA;
     }
     return CAT_OK;
 }
 
+// `tmOut`: tensor map of the 16-bit slab an epilogue stores through shared memory (tmap_out), or
+// NULL for epilogues that write their output directly.
 template <int A_MN, int B_MN, class Epi>
 int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& sched, const typename Epi::Params& ep,
-              int* status, int sm_count, cudaStream_t st) {
-    return cta_group() == 2 ? launch_tc_cg<A_MN, B_MN, Epi, 2>(tmA, tmB, sched, ep, status, sm_count, st)
-                            : launch_tc_cg<A_MN, B_MN, Epi, 1>(tmA, tmB, sched, ep, status, sm_count, st);
+              int* status, int sm_count, cudaStream_t st, const CUtensorMap* tmOut = nullptr) {
+    const CUtensorMap& o = tmOut ? *tmOut : tmA;
+    return cta_group() == 2 ? launch_tc_cg<A_MN, B_MN, Epi, 2>(tmA, tmB, o, sched, ep, status, sm_count, st)
+                            : launch_tc_cg<A_MN, B_MN, Epi, 1>(tmA, tmB, o, sched, ep, status, sm_count, st);
 }
 
 tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int band_m, int n_fastest) {
@@ -498,13 +506,15 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
         if (tmap_mn_major(&tmH_mn, Hs, rws, shape->d, shape->ldH) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_a(&tmZ_k, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
         if (tmap_mn_major(&tmZ_mn, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
+        CUtensorMap tmZ_out;
+        if (tmap_out(&tmZ_out, zs, rws, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
         if (kd) {   // logits of this row slab: softmax partials + label logit, logits kept as fp16
             const tc::Sched sched = make_sched(rws, shape->V, shape->d, S, band_tiles(shape->d), 0);
             tc::EpiFwdStore::Params ep;
             ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
             ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T; ep.ref = nullptr;
             ep.T = static_cast<int>(rws); ep.V = V;
-            const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+            const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmH_k, tmW_k, sched, ep, status, sm_count, st, &tmZ_out);
             if (rc != CAT_OK) return rc;
         } else {
             // per-row reference (the label logit), then the logits GEMM: softmax partials + label logit,
@@ -519,7 +529,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             ep.labels = y + r0; ep.part_m = part_m + r0; ep.part_l = part_l + r0; ep.z_label = z_label + r0;
             ep.zs = static_cast<__half*>(zs); ep.ldz = plan.ldz; ep.part_stride = T; ep.ref = ref + r0;
             ep.T = static_cast<int>(rws); ep.V = V;
-            const int rc = launch_tc<0, 0, tc::EpiFwdExp>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+            const int rc = launch_tc<0, 0, tc::EpiFwdExp>(tmH_k, tmW_k, sched, ep, status, sm_count, st, &tmZ_out);
             if (rc != CAT_OK) return rc;
             mark(st);
         }
@@ -543,7 +553,9 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
                 ep.z_label = reinterpret_cast<float*>(ws + kp.off_zt_label_t);
                 ep.zs = reinterpret_cast<__half*>(ws + kp.off_zt); ep.ldz = plan.ldz; ep.part_stride = kp.Ls_max; ep.ref = nullptr;
                 ep.T = static_cast<int>(t_span); ep.V = V;
-                const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmHt_k, tmWt_k, sched, ep, status, sm_count, st);
+                CUtensorMap tmZt_out;
+                if (tmap_out(&tmZt_out, ws + kp.off_zt, t_span, shape->V, plan.ldz) != CAT_OK) return CAT_ERR_CUDA;
+                const int rc = launch_tc<0, 0, tc::EpiFwdStore>(tmHt_k, tmWt_k, sched, ep, status, sm_count, st, &tmZt_out);
                 if (rc != CAT_OK) return rc;
                 rows::RowParams rp;
                 rp.part_m = ep.part_m; rp.part_l = ep.part_l; rp.z_label = ep.z_label; rp.labels = ep.labels;
@@ -830,7 +842,9 @@ static int bwd_core(const cat_shape* shape, const void* H, const void* W, const 
                 tc::EpiDz::Params ep;
                 ep.labels = y; ep.valid = valid; ep.lse = lse; ep.weight = weight; ep.dz = dz; ep.ld = plan.Vs;
                 ep.T = T; ep.V = V; ep.v0 = static_cast<int>(v0);
-                const int rc = launch_tc<0, 0, tc::EpiDz>(tmH_k, tmW_k, sched, ep, status, sm_count, st);
+                CUtensorMap tmDz_out;
+                if (tmap_out(&tmDz_out, dz, shape->T, width, plan.Vs) != CAT_OK) return CAT_ERR_CUDA;
+                const int rc = launch_tc<0, 0, tc::EpiDz>(tmH_k, tmW_k, sched, ep, status, sm_count, st, &tmDz_out);
                 if (rc != CAT_OK) return rc;
             }
             {   // dW[v0 : v0 + width, :] = (g/N) dz^T H

@@ -93,6 +93,46 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
     }
 }
 
+// Per-warp staging of 16-bit output tiles.  An epilogue thread owns one row, so a direct global
+// store makes every lane of a warp write a different row: 32 scattered 16-byte pieces per
+// instruction, which at a short contraction (d = 1024) held the logits GEMM at 70 % tensor
+// activity.  Instead the lanes write their pieces into a shared-memory tile of 32 rows x 64 columns
+// (128-byte rows, 128-byte swizzle, so the 8 lanes of a store phase hit different banks) and lane 0
+// sends the tile to global memory with one TMA store, which writes whole 128-byte lines and clips
+// rows / columns outside the tensor.  Two tiles per warp alternate; a tile is reused once the
+// store issued from it has read it (cp.async.bulk.wait_group.read).
+constexpr int OUT_TILE_BYTES = 32 * 128;
+constexpr int OUT_STAGE_BYTES = 4 * 2 * OUT_TILE_BYTES;      // four epilogue warps, two tiles each
+struct OutStage {
+    const CUtensorMap* tm;
+    uint32_t buf;      // shared-memory address of this warp's two tiles
+    int row0;          // tensor row of this warp's lane 0
+    int n_rows;        // rows of the tensor: a tile that starts at or past it is not sent
+    int lane;
+    int sel;
+    __device__ __forceinline__ void begin() {
+        if (lane == 0) ptx::tma_store_wait_read<1>();     // the store before last (same tile) has read it
+        __syncwarp();
+    }
+    // 16-byte piece `j` (0..7) of this lane's 128-byte row
+    __device__ __forceinline__ void put(int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+        ptx::st_shared_v4(buf + sel * OUT_TILE_BYTES + lane * 128 + ((j ^ (lane & 7)) << 4), a, b, c, d);
+    }
+    __device__ __forceinline__ void flush(int x) {
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < n_rows) {
+            ptx::tma_store_2d(tm, buf + sel * OUT_TILE_BYTES, x, row0);
+            ptx::tma_store_commit();
+        }
+        sel ^= 1;
+    }
+    __device__ __forceinline__ void finish() {
+        if (lane == 0) ptx::tma_store_wait_all();
+        __syncwarp();
+    }
+};
+
 // ------------------------------------------------------------------------------------------
 // Epilogues.  Each epilogue thread owns output row (m_tile*BM + row_in_tile) and walks the
 // 256 accumulator columns of a tile in chunks of 32 (one tcgen05.ld each).  taddr is the TMEM
@@ -143,12 +183,14 @@ struct EpiFwdT {
             if (STORE == 2) s.ref2 = p.ref[s.row] * LOG2E;
         }
     }
-    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr, OutStage& o) {
         const int col0 = n_tile * BN;
         const int ncols = min(BN, p.V - col0);
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
             if (c * 32 >= ncols) break;
+            const bool closes_pair = (c & 1) != 0 || (c + 1) * 32 >= ncols;   // last chunk of its 64-column staging tile
+            if (STORE != 0 && (c & 1) == 0) o.begin();
             uint32_t v[32];
             ptx::tmem_ld_32x32(taddr + c * 32, v);
             ptx::tmem_ld_wait();
@@ -162,18 +204,11 @@ struct EpiFwdT {
                     if (i >= live) f[i] = -INFINITY;
             }
             if (STORE == 1) {
-                if (s.row < p.T) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 pk;
-                        pk.x = ptx::pack_f16x2_sat(f[q * 8 + 0], f[q * 8 + 1]);
-                        pk.y = ptx::pack_f16x2_sat(f[q * 8 + 2], f[q * 8 + 3]);
-                        pk.z = ptx::pack_f16x2_sat(f[q * 8 + 4], f[q * 8 + 5]);
-                        pk.w = ptx::pack_f16x2_sat(f[q * 8 + 6], f[q * 8 + 7]);
-                        __stcs(dst + q, pk);
-                    }
-                }
+                for (int q = 0; q < 4; ++q)
+                    o.put((c & 1) * 4 + q, ptx::pack_f16x2_sat(f[q * 8 + 0], f[q * 8 + 1]), ptx::pack_f16x2_sat(f[q * 8 + 2], f[q * 8 + 3]),
+                          ptx::pack_f16x2_sat(f[q * 8 + 4], f[q * 8 + 5]), ptx::pack_f16x2_sat(f[q * 8 + 6], f[q * 8 + 7]));
+                if (closes_pair) o.flush(col0 + (c >> 1) * 64);
             }
             const int rel = s.y - (col0 + c * 32);
             if (rel >= 0 && rel < 32) {
@@ -212,12 +247,9 @@ struct EpiFwdT {
                 float s0, s1;
                 ptx::unpack_f32x2(sum2, s0, s1);
                 sum = s0 + s1;
-                if (s.row < p.T) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.zs + static_cast<size_t>(s.row) * p.ldz + col0 + c * 32);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        __stcs(dst + q, make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]));
-                }
+                for (int q = 0; q < 4; ++q) o.put((c & 1) * 4 + q, packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                if (closes_pair) o.flush(col0 + (c >> 1) * 64);
             } else {
                 const uint64_t l2e2 = ptx::pack_f32x2(LOG2E, LOG2E), nmb2 = ptx::pack_f32x2(-mb, -mb);
                 uint64_t sum2 = ptx::pack_f32x2(0.f, 0.f);
@@ -235,6 +267,7 @@ struct EpiFwdT {
             s.m_run = m_new;
         }
     }
+    __device__ static __forceinline__ int out_rows(const Params& p) { return STORE != 0 ? p.T : 0; }
     __device__ static __forceinline__ void end_item(const Params& p, const State& s, int group) {
         if (s.row < p.T) {
             p.part_m[static_cast<size_t>(group) * p.part_stride + s.row] = s.m_run;
@@ -280,12 +313,13 @@ struct EpiDz {
             }
         }
     }
-    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr, OutStage& o) {
         const int col0 = n_tile * BN;
         const int ncols = min(BN, p.V - p.v0 - col0);
-        __nv_bfloat16* out = p.dz + static_cast<size_t>(s.row) * p.ld + col0;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
+            if (c * 32 >= ncols) break;                     // columns past the vocabulary are never read back
+            if ((c & 1) == 0) o.begin();
             uint32_t v[32];
             ptx::tmem_ld_32x32(taddr + c * 32, v);
             ptx::tmem_ld_wait();
@@ -311,24 +345,14 @@ struct EpiDz {
                 for (int i = 0; i < 32; ++i)
                     if (i == rel) f[i] -= s.w;
             }
-            if (s.row < p.T) {
-                uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint4 pk;
-                    __nv_bfloat162 b0 = __floats2bfloat162_rn(f[q * 8 + 0], f[q * 8 + 1]);
-                    __nv_bfloat162 b1 = __floats2bfloat162_rn(f[q * 8 + 2], f[q * 8 + 3]);
-                    __nv_bfloat162 b2 = __floats2bfloat162_rn(f[q * 8 + 4], f[q * 8 + 5]);
-                    __nv_bfloat162 b3 = __floats2bfloat162_rn(f[q * 8 + 6], f[q * 8 + 7]);
-                    pk.x = *reinterpret_cast<uint32_t*>(&b0);
-                    pk.y = *reinterpret_cast<uint32_t*>(&b1);
-                    pk.z = *reinterpret_cast<uint32_t*>(&b2);
-                    pk.w = *reinterpret_cast<uint32_t*>(&b3);
-                    dst[q] = pk;
-                }
-            }
+            for (int q = 0; q < 4; ++q)
+                o.put((c & 1) * 4 + q, ptx::pack_bf16x2(f[q * 8 + 0], f[q * 8 + 1]), ptx::pack_bf16x2(f[q * 8 + 2], f[q * 8 + 3]),
+                      ptx::pack_bf16x2(f[q * 8 + 4], f[q * 8 + 5]), ptx::pack_bf16x2(f[q * 8 + 6], f[q * 8 + 7]));
+            if ((c & 1) != 0 || (c + 1) * 32 >= ncols) o.flush(col0 + (c >> 1) * 64);
         }
     }
+    __device__ static __forceinline__ int out_rows(const Params& p) { return p.T; }
     __device__ static __forceinline__ void end_item(const Params&, const State&, int) {}
 };
 
@@ -354,7 +378,7 @@ struct EpiOut {
         s.alpha = p.alpha ? *p.alpha : 1.f;
         if (p.row_scale && s.row < p.M) s.alpha *= p.row_scale[s.row];
     }
-    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr) {
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr, OutStage&) {
         const int col0 = n_tile * BN;
         const bool row_ok = s.row < p.M;
 #pragma unroll 1
@@ -406,6 +430,7 @@ struct EpiOut {
             }
         }
     }
+    __device__ static __forceinline__ int out_rows(const Params&) { return 0; }
     __device__ static __forceinline__ void end_item(const Params&, const State&, int) {}
 };
 
@@ -446,14 +471,15 @@ struct Geo {
     static constexpr int A_BYTES = A_STAGE_BYTES * KS;
     static constexpr int B_BYTES = B_SLICE_BYTES * KS;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+    static constexpr int SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
     static constexpr int TILE_M = BM * CG;                        // output rows per scheduled m-tile
 };
 
 template <int A_MN, int B_MN, class Epi, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const Sched sched, const typename Epi::Params ep, int* status) {
+            const __grid_constant__ CUtensorMap tmOut, const Sched sched, const typename Epi::Params ep, int* status) {
     using G = Geo<CG>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ Ctl ctl;
@@ -468,6 +494,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (threadIdx.x == 0) {
         ptx::prefetch_tmap(&tmA);
         ptx::prefetch_tmap(&tmB);
+        ptx::prefetch_tmap(&tmOut);
         for (int i = 0; i < G::STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctl.full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctl.empty[i]), 1);
@@ -624,16 +651,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         typename Epi::State st;
+        OutStage out;
+        out.tm = &tmOut;
+        out.buf = ring + G::RING_BYTES + static_cast<uint32_t>(quarter) * 2 * OUT_TILE_BYTES;
+        out.lane = lane;
+        out.sel = 0;
+        out.row0 = 0;
+        out.n_rows = Epi::out_rows(ep);
         for (int item = worker; item < sched.n_items && ok; item += n_workers) {
             int m_tile, group, n_begin, n_end;
             decode_item(sched, item, m_tile, group, n_begin, n_end);
             Epi::begin_item(ep, st, m_tile * CG + static_cast<int>(rank), row_in_tile);
+            out.row0 = (m_tile * CG + static_cast<int>(rank)) * BM + quarter * 32;
             for (int n = n_begin; n < n_end; ++n) {
                 ok = wait_bounded(ptx::smem_u32(&ctl.tfull[acc]), acc_phase, abort, status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after();
-                Epi::tile(ep, st, n, lane_base + acc * BN);
+                Epi::tile(ep, st, n, lane_base + acc * BN, out);
                 ptx::tc_fence_before();
                 if (CG == 1) {
                     ptx::mbar_arrive(ptx::smem_u32(&ctl.tempty[acc]));
@@ -646,6 +681,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             if (ok) Epi::end_item(ep, st, group);
         }
+        out.finish();      // the staged tiles have left shared memory before the CTA may exit
     }
 
     // Nothing of a pair may leave while its peer can still signal its barriers or read its
