@@ -311,14 +311,15 @@ EncodeTiledFn encode_fn() {
 
 // 2-D bf16 row-major tensor [rows][cols] with row pitch `ld` elements, 128-byte swizzle.
 // box = {box_cols (inner, 64 elements = 128 bytes), box_rows}.  Out-of-range elements read as zero.
-int make_tmap(CUtensorMap* m, const void* base, long long rows, long long cols, long long ld, int box_cols, int box_rows) {
+int make_tmap(CUtensorMap* m, const void* base, long long rows, long long cols, long long ld, int box_cols, int box_rows,
+              bool f32 = false) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return CAT_ERR_CUDA;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * (f32 ? 4 : 2)};
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    const CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? CAT_OK : CAT_ERR_CUDA;
@@ -342,6 +343,11 @@ inline int tmap_b(CUtensorMap* m, const void* base, long long mn, long long k, l
 // Output slab [rows][cols] of 16-bit values, written by the epilogue warps as boxes of 32 rows x 64 columns.
 inline int tmap_out(CUtensorMap* m, const void* base, long long rows, long long cols, long long ld) {
     return make_tmap(m, base, rows, cols, ld, 64, 32);
+}
+
+// fp32 output [rows][cols], written as boxes of 32 rows x 32 columns (128-byte rows).
+inline int tmap_out_f32(CUtensorMap* m, const void* base, long long rows, long long cols, long long ld) {
+    return make_tmap(m, base, rows, cols, ld, 32, 32, true);
 }
 
 int band_tiles(long long d) {
@@ -388,6 +394,21 @@ int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& s
     const CUtensorMap& o = tmOut ? *tmOut : tmA;
     return cta_group() == 2 ? launch_tc_cg<A_MN, B_MN, Epi, 2>(tmA, tmB, o, sched, ep, status, sm_count, st)
                             : launch_tc_cg<A_MN, B_MN, Epi, 1>(tmA, tmB, o, sched, ep, status, sm_count, st);
+}
+
+// Launch of a GEMM with the plain-output epilogue: fp32 outputs that either overwrite or accumulate in
+// place (pitch a multiple of 4 elements) take the staged TMA store / reduce-add route.
+template <int A_MN, int B_MN>
+int launch_out(const CUtensorMap& tmA, const CUtensorMap& tmB, const tc::Sched& sched, tc::EpiOut::Params ep, int* status,
+               int sm_count, cudaStream_t st) {
+    CUtensorMap tmO;
+    ep.staged = 0;
+    if (ep.out_f32 && !ep.add_bf16 && (ep.add_f32 == nullptr || ep.add_f32 == ep.out_f32) && ep.ld_out % 4 == 0 &&
+        !misaligned(ep.out_f32, 16)) {
+        if (tmap_out_f32(&tmO, ep.out_f32, ep.M, ep.N, ep.ld_out) != CAT_OK) return CAT_ERR_CUDA;
+        ep.staged = 1;
+    }
+    return launch_tc<A_MN, B_MN, tc::EpiOut>(tmA, tmB, sched, ep, status, sm_count, st, ep.staged ? &tmO : nullptr);
 }
 
 tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int band_m, int n_fastest) {
@@ -614,7 +635,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
             ep.alpha = scale; ep.M = static_cast<int>(rws); ep.N = d;
             if (!kd) ep.row_scale = a_row + r0;
             ep.out_bf16 = static_cast<__nv_bfloat16*>(dH) + r0 * shape->ldH; ep.ld_out = shape->ldH;
-            const int rc = launch_tc<0, 1, tc::EpiOut>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
+            const int rc = launch_out<0, 1>(tmZ_k, tmW_mn, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
             mark(st);
         }
@@ -639,7 +660,7 @@ int fused_core(const cat_shape* shape, const void* H, const void* W, const int64
                 if (last) { ep.out_bf16 = static_cast<__nv_bfloat16*>(dW); ep.ld_out = shape->ldW; }
                 else { ep.out_f32 = dw_acc; ep.ld_out = shape->d; }
             }
-            const int rc = launch_tc<1, 1, tc::EpiOut>(tmZ_mn, tmH_mn, sched, ep, status, sm_count, st);
+            const int rc = launch_out<1, 1>(tmZ_mn, tmH_mn, sched, ep, status, sm_count, st);
             if (rc != CAT_OK) return rc;
             mark(st);
         }
@@ -859,7 +880,7 @@ static int bwd_core(const cat_shape* shape, const void* H, const void* W, const 
                     ep.out_bf16 = static_cast<__nv_bfloat16*>(dW) + v0 * shape->ldW;
                     if (accumulate_dW) ep.add_bf16 = ep.out_bf16;
                 }
-                const int rc = launch_tc<1, 1, tc::EpiOut>(tmDz_mn, tmH_mn, sched, ep, status, sm_count, st);
+                const int rc = launch_out<1, 1>(tmDz_mn, tmH_mn, sched, ep, status, sm_count, st);
                 if (rc != CAT_OK) return rc;
                 if (slab_events && cudaEventRecord(static_cast<cudaEvent_t>(slab_events[sl]), st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
             }
@@ -871,7 +892,7 @@ static int bwd_core(const cat_shape* shape, const void* H, const void* W, const 
                 if (!first) { ep.add_f32 = dh_acc; ep.ld_add = shape->d; }
                 if (last) { ep.out_bf16 = static_cast<__nv_bfloat16*>(dH); ep.ld_out = shape->ldH; }
                 else { ep.out_f32 = dh_acc; ep.ld_out = shape->d; }
-                const int rc = launch_tc<0, 1, tc::EpiOut>(tmDz_k, tmW_mn, sched, ep, status, sm_count, st);
+                const int rc = launch_out<0, 1>(tmDz_k, tmW_mn, sched, ep, status, sm_count, st);
                 if (rc != CAT_OK) return rc;
             }
         } else {

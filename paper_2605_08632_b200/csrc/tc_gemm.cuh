@@ -118,11 +118,12 @@ struct OutStage {
     __device__ __forceinline__ void put(int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
         ptx::st_shared_v4(buf + sel * OUT_TILE_BYTES + lane * 128 + ((j ^ (lane & 7)) << 4), a, b, c, d);
     }
-    __device__ __forceinline__ void flush(int x) {
+    __device__ __forceinline__ void flush(int x, bool add = false) {
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0 && row0 < n_rows) {
-            ptx::tma_store_2d(tm, buf + sel * OUT_TILE_BYTES, x, row0);
+            if (add) ptx::tma_reduce_add_2d(tm, buf + sel * OUT_TILE_BYTES, x, row0);
+            else ptx::tma_store_2d(tm, buf + sel * OUT_TILE_BYTES, x, row0);
             ptx::tma_store_commit();
         }
         sel ^= 1;
@@ -368,6 +369,8 @@ struct EpiOut {
         __nv_bfloat16* out_bf16;       // [M][ld_out] or nullptr
         long long ld_add, ld_out;
         int M, N;
+        int staged;                    // 1: fp32 output, no addend or the output itself as addend: tiles of
+                                       //    32 x 32 go through shared memory and a TMA store / reduce-add
     };
     struct State {
         float alpha;
@@ -378,15 +381,24 @@ struct EpiOut {
         s.alpha = p.alpha ? *p.alpha : 1.f;
         if (p.row_scale && s.row < p.M) s.alpha *= p.row_scale[s.row];
     }
-    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr, OutStage&) {
+    __device__ static __forceinline__ void tile(const Params& p, State& s, int n_tile, uint32_t taddr, OutStage& o) {
         const int col0 = n_tile * BN;
         const bool row_ok = s.row < p.M;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
             if (col0 + c * 32 >= p.N) break;
+            if (p.staged) o.begin();
             uint32_t v[32];
             ptx::tmem_ld_32x32(taddr + c * 32, v);
             ptx::tmem_ld_wait();
+            if (p.staged) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    o.put(j, __float_as_uint(s.alpha * __uint_as_float(v[4 * j])), __float_as_uint(s.alpha * __uint_as_float(v[4 * j + 1])),
+                          __float_as_uint(s.alpha * __uint_as_float(v[4 * j + 2])), __float_as_uint(s.alpha * __uint_as_float(v[4 * j + 3])));
+                o.flush(col0 + c * 32, p.add_f32 != nullptr);
+                continue;
+            }
             if (!row_ok) continue;
             const int cbase = col0 + c * 32;
 #pragma unroll
@@ -430,7 +442,7 @@ struct EpiOut {
             }
         }
     }
-    __device__ static __forceinline__ int out_rows(const Params&) { return 0; }
+    __device__ static __forceinline__ int out_rows(const Params& p) { return p.staged ? p.M : 0; }
     __device__ static __forceinline__ void end_item(const Params&, const State&, int) {}
 };
 
