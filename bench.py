@@ -35,10 +35,10 @@ import torch
 # first row slab of the one-call path, ncu_two_call_gemms_config2.md for the two-call forward).
 # Valid for that kernel, workload and T only; None for anything else.
 TRAFFIC_BYTES = {
-    ("config2", 16384, "logits"): 797286000 + 2387855000,
-    ("config2", 16384, "dH"): 8383099000 + 38185000,
-    ("config2", 16384, "dW"): 4698015000 + 1037342000,
-    ("config2", 16384, "fwd_two_call"): 3495158272 + 20604672,
+    ("config2", 16384, "logits"): 972038000 + 2392758000,
+    ("config2", 16384, "dH"): 8332829000 + 36699000,
+    ("config2", 16384, "dW"): 4663208000 + 1036382000,
+    ("config2", 16384, "fwd_two_call"): 3061464832 + 21341440,
 }
 STAGES = ("label_ref", "logits", "rows", "slab_prep", "dH", "dW")
 STAGE_KERNEL = {
