@@ -226,3 +226,27 @@ def test_errors_on_gpu_box_leave_context_usable():
         B.cat_loss_fwd(s, x, x, x, None, None, x, x, x, x, None, x[:16])
     assert e.value.code == -5
     torch.cuda.synchronize()
+
+
+def test_single_cta_kernels_selected_by_environment_variable():
+    """CAT_LOSS_CTA_PAIR=0 selects the one-CTA 128x256 kernels (read once per process, hence the
+    child process); they must give the same answers within the same tolerances."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import sys; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+        "from paper_2605_08632_b200 import synth\n"
+        "from parity_util import run_gpu, run_gpu_fused, run_oracle, check_forward, check_backward\n"
+        "for cfg, kw in ((41, dict(T=1000, d=200, V=5000)), (3, dict(T=400))):\n"
+        "    b = synth.make_batch(cfg, **kw)\n"
+        "    fwd, dH, dW = run_oracle(b)\n"
+        "    for run in (run_gpu, run_gpu_fused):\n"
+        "        g = run(b, slab_mib=1 if cfg == 41 else 0)\n"
+        "        check_forward(g, fwd, b.K, b.torch_dtype, b.V)\n"
+        "        check_backward(g, fwd, dH, dW, b.K, b.torch_dtype)\n"
+        "print('single-cta ok')\n" % (root, os.path.join(root, "tests")))
+    env = dict(os.environ, CAT_LOSS_CTA_PAIR="0")
+    res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0 and "single-cta ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
