@@ -136,3 +136,41 @@ def test_window_edges_and_masked_positions():
     c = tc.conf_seq.cpu().numpy()
     ref, _ = O.target_confidence(batch.H, batch.W, y, valid)
     assert c[5] == c[9] == c[17] == 1.0 and np.allclose(c, ref, rtol=5e-3)
+
+
+def _golden(name):
+    import os
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append([p.strip() for p in line.split("|")])
+    return rows
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_scan_kernels_on_the_hand_examples(fused):
+    """The hand-evaluated instances of Eq. 10 and of the fixed decay (tests/golden/) through the CUDA
+    scan (warp-shuffle kernel for K a power of two, per-block kernel otherwise): supplied confidences,
+    exact dyadic products, so the weights must match to the bit."""
+    dev = "cuda"
+    for name, decay in (("eq10_hand_examples.txt", False), ("fixed_decay_hand_examples.txt", True)):
+        for K, a, v, w in _golden(name):
+            K = int(K)
+            valid = torch.tensor([int(x) for x in v.split()], dtype=torch.uint8)
+            expect = np.array(w.split(), dtype=np.float32)
+            reps = 3                                         # a few blocks, so lanes of several blocks share a warp
+            batch = synth.make_batch(2, T=K * reps, d=64, V=256, K=K)
+            kw = dict(fixed_decay_gamma=float(a)) if decay else {}
+            cl = CatLoss(batch.T, batch.d, batch.V, K, **kw)
+            ce = None if decay else torch.tensor([float(x) for x in a.split()] * reps, dtype=torch.float32, device=dev)
+            args = (batch.H.to(dev), batch.W.to(dev), batch.labels.to(dev), valid.repeat(reps).to(dev))
+            if fused:
+                cl.forward_backward(*args, conf_ext=ce)
+            else:
+                cl.forward(*args, ce)
+            torch.cuda.synchronize()
+            got = cl.weight.cpu().numpy().reshape(reps, K)
+            for r in range(reps):
+                assert got[r].tobytes() == expect.tobytes(), (name, K, a, v, got[r], expect)
