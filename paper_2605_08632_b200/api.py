@@ -142,3 +142,45 @@ class TargetConfidence:
 
     def status(self) -> int:
         return int(self.ws[:4].view(torch.int32).item())
+
+
+class _CatLossFn(torch.autograd.Function):
+    """autograd glue: the loss and both gradients come out of one cat_loss_fwd_bwd call in forward();
+    backward() hands them over, multiplied by the incoming scalar gradient when that is not 1."""
+
+    @staticmethod
+    def forward(ctx, H, W, labels, valid, conf_ext, K, engine):
+        loss, dH, dW = engine.forward_backward(H.detach(), W.detach(), labels, valid, conf_ext=conf_ext)
+        ctx.save_for_backward(dH, dW)
+        return loss.clone().reshape(())
+
+    @staticmethod
+    def backward(ctx, grad_out):
+        dH, dW = ctx.saved_tensors
+        if bool((grad_out == 1).item()):
+            return dH, dW, None, None, None, None, None
+        return dH * grad_out.to(dH.dtype), dW * grad_out.to(dW.dtype), None, None, None, None, None
+
+
+class CatLossModule(torch.nn.Module):
+    """Drop-in loss head for a draft-model training loop: `loss = head(H, labels, valid)` with
+    H [T, d] the hidden states of the draft positions (T = blocks * K), using `weight` [V, d] as the
+    LM head.  The library's dW is float32; autograd casts it to the parameter's dtype when it stores
+    it in `weight.grad`.  An upstream gradient other than 1 is applied by a tensor multiply in
+    backward() (chain-rule glue; pass `grad_loss` to CatLoss.forward_backward to have the kernels
+    apply a scale instead).  One engine (buffers for one T) is kept per distinct T."""
+
+    def __init__(self, weight: torch.Tensor, K: int, slab_mib: int = 0):
+        super().__init__()
+        self.weight = weight if isinstance(weight, torch.nn.Parameter) else torch.nn.Parameter(weight)
+        self.K = K
+        self.slab_mib = slab_mib
+        self._engines = {}
+
+    def forward(self, H, labels, valid=None, conf_ext=None):
+        T, d = H.shape
+        eng = self._engines.get(T)
+        if eng is None:
+            eng = self._engines[T] = CatLoss(T, d, self.weight.shape[0], self.K, dtype=H.dtype, slab_mib=self.slab_mib,
+                                             device=str(H.device))
+        return _CatLossFn.apply(H, self.weight, labels, valid, conf_ext, self.K, eng)

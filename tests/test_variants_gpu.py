@@ -174,3 +174,20 @@ def test_scan_kernels_on_the_hand_examples(fused):
             got = cl.weight.cpu().numpy().reshape(reps, K)
             for r in range(reps):
                 assert got[r].tobytes() == expect.tobytes(), (name, K, a, v, got[r], expect)
+
+
+def test_autograd_module_matches_oracle_and_scales_with_the_upstream_gradient():
+    from paper_2605_08632_b200.api import CatLossModule
+    batch = synth.make_batch(41, T=512, d=256, V=4000)
+    dev = "cuda"
+    W = batch.W.to(dev).clone().requires_grad_(True)
+    H = batch.H.to(dev).clone().requires_grad_(True)
+    head = CatLossModule(W, batch.K)
+    loss = head(H, batch.labels.to(dev), batch.valid.to(dev))
+    (0.5 * loss).backward()
+    torch.cuda.synchronize()
+    fwd, dH, dW = O.cat_forward_backward(batch.H, batch.W, batch.labels, batch.valid, batch.K, g=0.5)
+    assert abs(loss.item() - fwd["loss"]) <= 1e-3 * fwd["loss"]
+    assert H.grad.dtype == torch.bfloat16 and head.weight.grad is not None
+    assert rel_l2(H.grad.float().cpu().numpy(), dH) <= 1.2e-2          # one more bf16 rounding from the scaling by 0.5
+    assert rel_l2(head.weight.grad.float().cpu().numpy(), dW) <= 1.2e-2
