@@ -127,6 +127,14 @@ def test_row_pitch_larger_than_d():
     assert rel_l2(cl.dH[:, :192].float().cpu().numpy(), dH) <= 1e-2
     assert rel_l2(cl.dW[:, :192].cpu().numpy(), dW) <= 1e-2
     assert torch.all(cl.dH[:, 192:] == 3.0) and torch.all(cl.dW[:, 192:] == 3.0)
+    # the one-call path on the same pitched buffers
+    cl.dH.fill_(3.0); cl.dW.fill_(3.0)
+    cl.forward_backward(Hp, Wp, labels, valid)
+    torch.cuda.synchronize()
+    assert cl.fused_status() == 0 and abs(cl.loss.item() - fwd["loss"]) <= 1e-3 * fwd["loss"]
+    assert rel_l2(cl.dH[:, :192].float().cpu().numpy(), dH) <= 1e-2
+    assert rel_l2(cl.dW[:, :192].cpu().numpy(), dW) <= 1e-2
+    assert torch.all(cl.dH[:, 192:] == 3.0) and torch.all(cl.dW[:, 192:] == 3.0)
 
 
 # ---------------------------------------------------------------- fused forward+backward (no recompute)
