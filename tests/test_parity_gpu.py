@@ -258,3 +258,21 @@ def test_single_cta_kernels_selected_by_environment_variable():
     env = dict(os.environ, CAT_LOSS_CTA_PAIR="0")
     res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
     assert res.returncode == 0 and "single-cta ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
+
+
+def test_seeded_random_shapes_both_paths():
+    """Twelve seeded random problem shapes (rows, hidden size, vocabulary, block length, slab cap all
+    drawn, masks on) through both paths: ragged tiles in every dimension and odd slab boundaries."""
+    rng = np.random.default_rng(20240611)
+    for _ in range(12):
+        K = int(rng.choice([1, 2, 3, 4, 6, 8, 16, 32]))
+        blocks = int(rng.integers(1, 1 + 1200 // K))
+        d = 8 * int(rng.integers(1, 80))
+        V = int(rng.integers(2, 9000))
+        slab = int(rng.choice([0, 1, 2, 3]))
+        batch = synth.make_batch(41, T=K * blocks, d=d, V=V, K=K)
+        fwd, dH, dW = run_oracle(batch)
+        for run in (run_gpu, run_gpu_fused):
+            gpu = run(batch, slab_mib=slab)
+            check_forward(gpu, fwd, K, batch.torch_dtype, V)
+            check_backward(gpu, fwd, dH, dW, K, batch.torch_dtype, per_position=False)
