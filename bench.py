@@ -418,7 +418,7 @@ def main():
     out["launches_per_step"] = per_step
 
     if not args.no_cpu_baseline:
-        rows = 512
+        rows = 2048            # about 10 s of fp64 work on 16 host cores
         rate, ms = oracle_sample_rate(batch, rows)
         out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                                "sample": f"first {rows} rows (whole K-blocks) of the workload, fwd+bwd incl. their dW contribution, {ms:.0f} ms"}
