@@ -366,8 +366,7 @@ int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorM
     }
     const int workers = sm_count / CG;
     const int grid = CG * (sched.n_items < workers ? sched.n_items : workers);
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
     cfg.blockDim = dim3(tc::NUM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = smem;
