@@ -24,7 +24,9 @@
  * General conventions
  *   - Every data pointer is a DEVICE pointer owned by the caller, valid on the current
  *     device, unless a parameter says "host".  cat_shape is read on the host.
- *   - Nothing is allocated or freed here and no state is kept between calls.
+ *   - Nothing is allocated or freed here and no state is kept between calls.  The one exception is
+ *     cat_loss_fwd_static, which owns a fixed device array inside the library image and remembers,
+ *     per device, that array's address (see there).
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *     stream) and the call returns without synchronising.
  *   - Argument errors that the host can see return a negative cat_status before anything is
@@ -268,6 +270,9 @@ int cat_loss_fused_slabs(const cat_shape* shape, int64_t* row_begin, int capacit
  *   - All calls share the one array and it keeps whatever the last call left in it; the
  *     words that must start at zero are cleared by every call.  Two calls whose GPU work
  *     overlaps (different streams, or different host threads) race on it: serialise them.
+ *   - The device status word of this call sits in the built-in array, out of the caller's reach:
+ *     pass `stats` to see it (cat_stats.device_status); with stats == NULL a timed-out wait inside
+ *     a kernel goes unreported.
  */
 #define CAT_STATIC_SCRATCH_BYTES (32u << 20)
 int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W,
@@ -360,8 +365,11 @@ size_t cat_kd_workspace_bytes(const cat_shape* shape, const cat_kd_desc* desc, c
  *   desc              target-side sizes, beta, confidence source                        (host, in)
  *   Ht, Wt            [L, d_t], [V, d_t] bf16 target hidden states and target LM head    (device, in)
  *   block_start_host  [T/K] int64, HOST pointer, non-decreasing: sequence position of each block's
- *                     first drafted token.  Copied to the device inside the call (one
- *                     cudaMemcpyAsync on the stream); the caller may reuse it on return.
+ *                     first drafted token.  Read on the host during the call (slab planning) and
+ *                     copied to the device by one cudaMemcpyAsync on the stream: keep the array
+ *                     unchanged until the stream has passed that copy (for pageable memory that is
+ *                     when the call returns, for pinned memory it is not), and do not make this
+ *                     call while the stream is being captured.
  *   conf_ext          [T] fp32 or NULL                                                   (device, in)
  *   loss              [3] fp32: total, its cross-entropy part (1/N) sum w CE, its distillation
  *                     part (1/N) sum w KD; total = beta * loss[1] + loss[2]              (device, out)
@@ -382,6 +390,26 @@ int cat_kd_loss_fwd_bwd(const cat_shape* shape, const cat_kd_desc* desc, const v
  * pass.  Host-only; returns 0 for an invalid shape.
  */
 int cat_loss_launch_count(const cat_shape* shape, int pass);
+
+/*
+ * Self-test of the error path that cat_stats.device_status / the workspace status word report (no
+ * counterpart in the paper: it concerns this library's kernels only).  Every wait inside the
+ * tensor-core kernels is bounded; one that runs out raises an abort flag that the other warp roles
+ * of the CTA watch, records CAT_ERR_TIMEOUT, and the CTA (or CTA pair) leaves through the normal
+ * teardown.  This call runs exactly that sequence -- the GEMM kernel's set-up, role split, bounded
+ * waits, abort flag and teardown -- in one CTA (or one pair, as the GEMMs are configured) with no
+ * copy and no tensor-core work in flight, around barriers that nothing signals:
+ *   role        0 = the TMA-producer lane, 1 = the MMA-issuing lane, 2 = the epilogue warps: the role
+ *               whose wait gets the limit short_ns; the others get long_ns and must leave early,
+ *               through the abort flag
+ *   short_ns    1 .. 1e8 (0.1 s);  long_ns  short_ns .. 5e9: anything else is CAT_ERR_SHAPE
+ *   status      [1] int32: cleared by the call, CAT_ERR_TIMEOUT once the kernel has run  (device, out)
+ *   elapsed_ns  [12] uint64, entry cta * 6 + warp: nanoseconds that warp waited; bit 63 is set if
+ *               its wait was (wrongly) satisfied; one CTA writes 6 entries, a pair 12     (device, out)
+ * The kernel returns by itself after about short_ns; nothing traps and the context stays usable.
+ */
+int cat_selftest_wait_timeout(int role, uint64_t short_ns, uint64_t long_ns, int32_t* status,
+                              uint64_t* elapsed_ns, void* cuda_stream);
 
 /* Static, NUL-terminated description of a cat_status value (host pointer, never freed). */
 const char* cat_status_string(int status);

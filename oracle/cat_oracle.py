@@ -58,6 +58,7 @@ __all__ = [
     "target_confidence",
     "window_confidence",
     "cat_forward",
+    "cat_forward_from_row_stats",
     "cat_backward",
     "cat_forward_backward",
     "cat_dH_rows",
@@ -228,6 +229,14 @@ def cat_forward(H, W, labels, valid, K: int, conf_ext=None, row_chunk: int = 102
             p_sum = np.exp(z - lse[r0:r1, None]).sum(axis=1)
             assert np.all(np.abs(p_sum - 1.0) <= 1e-12), "softmax rows do not sum to 1"
         zy[r0:r1] = z[np.arange(r1 - r0), ysafe[r0:r1]]
+    return cat_forward_from_row_stats(lse, zy, y, valid, K, V, conf_ext=conf_ext, fixed_decay_gamma=fixed_decay_gamma)
+
+
+def cat_forward_from_row_stats(lse, z_label, labels, valid, K: int, V: int, conf_ext=None, fixed_decay_gamma=None) -> dict:
+    """Eq. 9-11 once the per-row log-partition lse[T] and label logit z_label[T] are known (the
+    second half of cat_forward; also used to rebuild a forward state from stored lse / z_label)."""
+    lse, zy, y = np.asarray(lse, dtype=np.float64), np.asarray(z_label, dtype=np.float64), _as_i64(labels)
+    ok = effective_valid(y, valid, V)
     p_label = np.exp(zy - lse)                      # probability of the label token
     if conf_ext is None:
         conf = np.where(ok, p_label, 1.0)           # Eq. 9 evaluated with this head

@@ -146,11 +146,14 @@ class TargetConfidence:
 
 class _CatLossFn(torch.autograd.Function):
     """autograd glue: the loss and both gradients come out of one cat_loss_fwd_bwd call in forward();
-    backward() hands them over, multiplied by the incoming scalar gradient when that is not 1."""
+    backward() hands them over, multiplied by the incoming scalar gradient when that is not 1.
+    The gradient buffers the call wrote become the graph node's own and the engine gets fresh ones,
+    so a second call through the same engine before backward() cannot overwrite them."""
 
     @staticmethod
     def forward(ctx, H, W, labels, valid, conf_ext, K, engine):
         loss, dH, dW = engine.forward_backward(H.detach(), W.detach(), labels, valid, conf_ext=conf_ext)
+        engine.dH, engine.dW = torch.empty_like(dH), torch.empty_like(dW)
         ctx.save_for_backward(dH, dW)
         return loss.clone().reshape(())
 

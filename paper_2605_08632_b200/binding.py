@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.cat_kd_workspace_bytes.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc), vp]
         L.cat_kd_loss_fwd_bwd.restype = ctypes.c_int
         L.cat_kd_loss_fwd_bwd.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc)] + [vp] * 16 + [ctypes.c_int, vp, sz, vp]
+        L.cat_selftest_wait_timeout.restype = ctypes.c_int
+        L.cat_selftest_wait_timeout.argtypes = [ctypes.c_int, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -263,6 +265,14 @@ def cat_kd_loss_fwd_bwd(shape, desc, H, W, labels, valid, Ht, Wt, block_start_ho
                                    workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_kd_loss_fwd_bwd")
+
+
+def cat_selftest_wait_timeout(role: int, short_ns: int, long_ns: int, status, elapsed_ns) -> None:
+    """Runs the kernels' time-out path on purpose (a bounded wait that nothing satisfies);
+    `status` int32[1] and `elapsed_ns` int64[12] are CUDA tensors written by the kernel."""
+    rc = lib().cat_selftest_wait_timeout(int(role), int(short_ns), int(long_ns), _ptr(status), _ptr(elapsed_ns), _stream())
+    if rc != CAT_OK:
+        raise CatError(rc, "cat_selftest_wait_timeout")
 
 
 def read_stats(stats_tensor: torch.Tensor) -> cat_stats:

@@ -419,6 +419,7 @@ tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int b
     s.band_m = band_m < 1 ? 1 : band_m;
     s.n_fastest = n_fastest;
     s.n_items = s.num_m_tiles * s.n_groups;
+    s.wait_ns = tc::WAIT_LIMIT_NS;
     return s;
 }
 
@@ -1110,6 +1111,50 @@ int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W, co
     // in the scratch is fully rewritten before it is read
     return cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, scratch,
                         static_cast<size_t>(CAT_STATIC_SCRATCH_BYTES), cuda_stream);
+}
+
+}  // extern "C"
+
+// Self-test of the kernels' time-out path: one CTA (or one CTA pair, as the GEMMs are configured) runs the
+// GEMM kernel's set-up, role split and teardown around waits that nothing will ever satisfy.
+template <int CG>
+static int launch_wait_probe(int role, unsigned long long short_ns, unsigned long long long_ns, int* status,
+                             unsigned long long* elapsed, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(CG, 1, 1);
+    cfg.blockDim = dim3(tc::NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, tc::wait_probe_kernel<CG>, role, short_ns, long_ns, status, elapsed) != cudaSuccess) {
+        cudaGetLastError();
+        return CAT_ERR_CUDA;
+    }
+    return CAT_OK;
+}
+
+extern "C" {
+
+int cat_selftest_wait_timeout(int role, uint64_t short_ns, uint64_t long_ns, int32_t* status, uint64_t* elapsed_ns,
+                              void* cuda_stream) {
+    if (!status || !elapsed_ns) return CAT_ERR_NULL;
+    if (role < 0 || role > 2 || short_ns == 0 || short_ns > 100000000ull || long_ns < short_ns || long_ns > 5000000000ull)
+        return CAT_ERR_SHAPE;
+    if (misaligned(status, 4) || misaligned(elapsed_ns, 8)) return CAT_ERR_ALIGN;
+    int sms = 0;
+    const int dc = check_device(&sms);
+    if (dc != CAT_OK) return dc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t), st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    unsigned long long* el = reinterpret_cast<unsigned long long*>(elapsed_ns);
+    return cta_group() == 2 ? launch_wait_probe<2>(role, short_ns, long_ns, status, el, st)
+                            : launch_wait_probe<1>(role, short_ns, long_ns, status, el, st);
 }
 
 }  // extern "C"

@@ -31,7 +31,8 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int MN_ATOM_BYTES = 64 * BK * 2;                // one 64(MN) x BK box of an MN-major operand
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // default limit of a wait (Sched::wait_ns)
+constexpr unsigned long long DRAIN_LIMIT_NS = 20000000ull;    // after an abort: how long issued copies / MMAs get to land
 constexpr int STATUS_TIMEOUT = -8;                        // CAT_ERR_TIMEOUT
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -44,6 +45,7 @@ struct Sched {
     int band_m;        // m-tiles per band when m runs fastest (keeps a band of A rows L2-resident)
     int n_fastest;     // 1: items ordered group-fastest within an m-tile; 0: m-fastest within (band, group)
     int n_items;       // num_m_tiles * n_groups
+    unsigned long long wait_ns;   // limit of every mbarrier wait in the kernel
 };
 
 __device__ __forceinline__ void decode_item(const Sched& s, int item, int& m_tile, int& group, int& n_begin, int& n_end) {
@@ -72,21 +74,28 @@ struct Ctl {
     volatile int abort;
 };
 
+// Waits for phase `parity` of an mbarrier, at most `limit_ns`.  A wait that runs out raises the CTA's abort
+// flag and records CAT_ERR_TIMEOUT; a wait that sees the flag raised by another role gives up at once.
+// DRAIN = true is for the clean-up after an abort: the flag is already up, so it is neither heeded nor
+// set, and the wait simply ends when the barrier completes or the limit passes.
+template <bool DRAIN = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort, int* status,
-                                             unsigned long long limit_ns = WAIT_LIMIT_NS) {
+                                             unsigned long long limit_ns) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
     uint32_t spins = 0;
     while (true) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
-            if (*abort) return false;
+            if (!DRAIN && *abort) return false;
             const unsigned long long now = ptx::globaltimer_ns();
             if (t0 == 0) {
                 t0 = now;
             } else if (now - t0 > limit_ns) {
-                *abort = 1;
-                atomicExch(status, STATUS_TIMEOUT);
+                if (!DRAIN) {
+                    *abort = 1;
+                    atomicExch(status, STATUS_TIMEOUT);
+                }
                 return false;
             }
         }
@@ -488,26 +497,12 @@ struct Geo {
     static constexpr int TILE_M = BM * CG;                        // output rows per scheduled m-tile
 };
 
-template <int A_MN, int B_MN, class Epi, int CG>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const __grid_constant__ CUtensorMap tmOut, const Sched sched, const typename Epi::Params ep, int* status) {
-    using G = Geo<CG>;
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ Ctl ctl;
-    const uint32_t ring = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-    const uint32_t rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
-    const bool leader = rank == 0;
-    const int worker = blockIdx.x / CG;          // a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
-    const int n_workers = gridDim.x / CG;
-
+// Set-up shared by every CTA of the kernels below: barriers, the abort flag, TMEM (warp 1 owns it).
+// On return the barriers exist in both CTAs of a pair and ctl.tmem_base is valid.
+template <int CG>
+__device__ __forceinline__ void cta_begin(Ctl& ctl, int n_stages, int warp) {
     if (threadIdx.x == 0) {
-        ptx::prefetch_tmap(&tmA);
-        ptx::prefetch_tmap(&tmB);
-        ptx::prefetch_tmap(&tmOut);
-        for (int i = 0; i < G::STAGES; ++i) {
+        for (int i = 0; i < n_stages; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctl.full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctl.empty[i]), 1);
         }
@@ -532,8 +527,46 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (CG == 1) __syncthreads();
     else ptx::cluster_sync_all();     // the peer's barriers must exist before anything signals them
     ptx::tc_fence_after();
+}
+
+// Teardown, also after an abort.  Nothing of a pair may leave while its peer can still signal its
+// barriers or read its shared memory, so the pair meets here before TMEM is returned.
+template <int CG>
+__device__ __forceinline__ void cta_end(int warp, uint32_t tmem) {
+    ptx::tc_fence_before();
+    if (CG == 1) __syncthreads();
+    else ptx::cluster_sync_all();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        if (CG == 1) ptx::tmem_dealloc<TMEM_COLS>(tmem);
+        else ptx::tmem_dealloc_pair<TMEM_COLS>(tmem);
+    }
+}
+
+template <int A_MN, int B_MN, class Epi, int CG>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmOut, const Sched sched, const typename Epi::Params ep, int* status) {
+    using G = Geo<CG>;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ Ctl ctl;
+    const uint32_t ring = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
+    const int worker = blockIdx.x / CG;          // a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
+    const int n_workers = gridDim.x / CG;
+
+    if (threadIdx.x == 0) {
+        ptx::prefetch_tmap(&tmA);
+        ptx::prefetch_tmap(&tmB);
+        ptx::prefetch_tmap(&tmOut);
+    }
+    cta_begin<CG>(ctl, G::STAGES, warp);
     const uint32_t tmem = ctl.tmem_base;
     volatile int* abort = &ctl.abort;
+    const unsigned long long wait_ns = sched.wait_ns;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -547,7 +580,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int n = n_begin; n < n_end && ok; ++n) {
                     const int n0 = n * BN + static_cast<int>(rank) * G::BN_CTA;
                     for (int kb = 0; kb < sched.num_kb; ++kb) {
-                        if (!wait_bounded(ptx::smem_u32(&ctl.empty[stage]), phase ^ 1u, abort, status)) { ok = false; break; }
+                        if (!wait_bounded(ptx::smem_u32(&ctl.empty[stage]), phase ^ 1u, abort, status, wait_ns)) { ok = false; break; }
                         const uint32_t full_local = ptx::smem_u32(&ctl.full[stage]);
                         if (leader) ptx::mbar_arrive_expect_tx(full_local, G::STAGE_BYTES * CG);
                         const uint32_t full_sig = CG == 1 ? full_local : ptx::mapa_shared(full_local, 0);   // pair: the leader's barrier
@@ -581,11 +614,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const uint32_t back = issued < G::STAGES ? issued : G::STAGES;
                     for (uint32_t i = 0; i < back; ++i) {
                         const uint32_t q = issued - 1 - i;
-                        wait_bounded(ptx::smem_u32(&ctl.full[q % G::STAGES]), (q / G::STAGES) & 1u, abort, status, 20000000ull);
+                        wait_bounded<true>(ptx::smem_u32(&ctl.full[q % G::STAGES]), (q / G::STAGES) & 1u, abort, status, DRAIN_LIMIT_NS);
                     }
                 } else {
                     const unsigned long long t0 = ptx::globaltimer_ns();
-                    while (ptx::globaltimer_ns() - t0 < 20000000ull) __nanosleep(1000);
+                    while (ptx::globaltimer_ns() - t0 < DRAIN_LIMIT_NS) __nanosleep(1000);
                 }
             }
         }
@@ -614,11 +647,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 int m_tile, group, n_begin, n_end;
                 decode_item(sched, item, m_tile, group, n_begin, n_end);
                 for (int n = n_begin; n < n_end && ok; ++n) {
-                    if (!wait_bounded(ptx::smem_u32(&ctl.tempty[acc]), acc_phase ^ 1u, abort, status)) { ok = false; break; }
+                    if (!wait_bounded(ptx::smem_u32(&ctl.tempty[acc]), acc_phase ^ 1u, abort, status, wait_ns)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem + acc * BN;
                     for (int kb = 0; kb < sched.num_kb; ++kb) {
-                        if (!wait_bounded(full0 + stage * 8u, phase, abort, status)) { ok = false; break; }
+                        if (!wait_bounded(full0 + stage * 8u, phase, abort, status, wait_ns)) { ok = false; break; }
                         ptx::tc_fence_after();
 #pragma unroll
                         for (int h = 0; h < G::KS; ++h) {
@@ -651,7 +684,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 // aborted: make sure no MMA is still in flight before TMEM is freed
                 if (CG == 1) ptx::umma_commit(ptx::smem_u32(&ctl.drain));
                 else ptx::umma_commit_pair(ptx::smem_u32(&ctl.drain), 1);
-                wait_bounded(ptx::smem_u32(&ctl.drain), 0, abort, status, 20000000ull);
+                wait_bounded<true>(ptx::smem_u32(&ctl.drain), 0, abort, status, DRAIN_LIMIT_NS);
             }
         }
         __syncwarp();
@@ -676,7 +709,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             Epi::begin_item(ep, st, m_tile * CG + static_cast<int>(rank), row_in_tile);
             out.row0 = (m_tile * CG + static_cast<int>(rank)) * BM + quarter * 32;
             for (int n = n_begin; n < n_end; ++n) {
-                ok = wait_bounded(ptx::smem_u32(&ctl.tfull[acc]), acc_phase, abort, status);
+                ok = wait_bounded(ptx::smem_u32(&ctl.tfull[acc]), acc_phase, abort, status, wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after();
@@ -696,16 +729,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         out.finish();      // the staged tiles have left shared memory before the CTA may exit
     }
 
-    // Nothing of a pair may leave while its peer can still signal its barriers or read its
-    // shared memory, so the pair meets here before TMEM is returned.
-    ptx::tc_fence_before();
-    if (CG == 1) __syncthreads();
-    else ptx::cluster_sync_all();
-    if (warp == 1) {
-        ptx::tc_fence_after();
-        if (CG == 1) ptx::tmem_dealloc<TMEM_COLS>(tmem);
-        else ptx::tmem_dealloc_pair<TMEM_COLS>(tmem);
+    cta_end<CG>(warp, tmem);
+}
+
+// ------------------------------------------------------------------------------------------
+// Test hook for the time-out path: the set-up, the role split, the abort flag and the teardown of
+// gemm_kernel (same functions), with no copy and no MMA in flight.  Every role waits on a barrier
+// that nothing ever signals: role `which` (0 = producer lane, 1 = MMA lane, 2 = epilogue warps) with
+// the limit `short_ns`, the others with `long_ns`.  The short wait runs out, raises the CTA's abort
+// flag and writes CAT_ERR_TIMEOUT to *status; the other roles must then leave through the flag long
+// before their own limit.  elapsed_ns[cta * 6 + warp] reports how long each warp waited.  The kernel
+// returns by itself; nothing traps and nothing is left waiting.
+// ------------------------------------------------------------------------------------------
+template <int CG>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+wait_probe_kernel(int which, unsigned long long short_ns, unsigned long long long_ns, int* status, unsigned long long* elapsed_ns) {
+    __shared__ Ctl ctl;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    cta_begin<CG>(ctl, 1, warp);
+    const uint32_t tmem = ctl.tmem_base;
+    volatile int* abort = &ctl.abort;
+    const unsigned long long t0 = ptx::globaltimer_ns();
+    const int role = warp < 2 ? warp : 2;
+    const unsigned long long limit = role == which ? short_ns : long_ns;
+    bool ok = true;
+    if (warp == 0) {
+        if (lane == 0) ok = wait_bounded(ptx::smem_u32(&ctl.empty[0]), 0, abort, status, limit);
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) ok = wait_bounded(ptx::smem_u32(&ctl.full[0]), 0, abort, status, limit);
+        __syncwarp();
+    } else {
+        ok = wait_bounded(ptx::smem_u32(&ctl.tfull[0]), 0, abort, status, limit);
+        ok = __all_sync(0xffffffffu, ok);
     }
+    if (lane == 0) elapsed_ns[blockIdx.x * (NUM_THREADS / 32) + warp] = (ptx::globaltimer_ns() - t0) | (ok ? (1ull << 63) : 0ull);
+    cta_end<CG>(warp, tmem);
 }
 
 }  // namespace tc

@@ -1,13 +1,26 @@
-"""Full-size parity in the launch configuration bench.py times (default slab sizes).
+"""Full-size parity for every bf16 configuration, in the launch configuration bench.py times
+(default slab sizes), on both entry-point paths: cat_loss_fwd + cat_loss_bwd and cat_loss_fwd_bwd.
 
-The oracle cannot afford every output at these sizes, so it computes sampled ones exactly:
-whole draft blocks (lse, confidence, weight and the dH rows of those blocks) for configs 2-5,
-and for config 2, the benchmark workload, the whole forward pass (exact loss, every lse and
-weight) plus sampled dW rows.  On top come properties that hold at any size: the weights are
-the binary32 product of the GPU's own confidences for every row, dW sums to zero over the
-vocabulary, masked rows have zero dH, and the loss equals the fp64 reduction of the per-row
-outputs.  Both entry-point paths are checked: cat_loss_fwd + cat_loss_bwd and cat_loss_fwd_bwd.
+What the oracle supplies at these sizes:
+  * its forward pass over EVERY row (tests/golden/fullsize_forward_cfg<N>.npz, written by
+    tests/golden/make_fullsize_forward.py from the oracle alone; recomputed here when the seeded
+    inputs drawn on this machine do not have the stored digests): every row's lse, confidence and
+    weight and the exact loss are compared;
+  * dH of >= 64 seeded whole draft blocks per configuration, forced to include masked blocks
+    (block-end tails, mid-block holes, fully masked), biased rows, the first and the last block;
+  * >= 256 rows of dW per configuration.  dW[v, :] sums over all rows, so with the whole forward
+    state the oracle evaluates any row of it exactly; forced to include the 28 most frequent labels
+    (with Zipf labels a few token ids receive most one-hot terms), ids no row is labelled with, ids 0
+    and V - 1, and the ids of the ragged last vocabulary tile.  This is the check on the fp32
+    accumulation of dW over the row slabs of the one-call path and over the vocabulary slabs of
+    the two-call path.
+On top come properties that hold at any size: the weights are the binary32 product of the GPU's
+own confidences for every row, dW sums to zero over the vocabulary, masked rows have zero dH.
 """
+import os
+import sys
+import warnings
+
 import numpy as np
 import pytest
 import torch
@@ -16,63 +29,85 @@ from oracle import cat_oracle as O
 from paper_2605_08632_b200 import synth
 from paper_2605_08632_b200.api import CatLoss
 
-from parity_util import TOL, rel_l2
+from parity_util import POSITION_FACTOR, TOL, check_dH_rows_by_position, rel_l2
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+if GOLDEN not in sys.path:
+    sys.path.insert(0, GOLDEN)
+import make_fullsize_forward as G  # noqa: E402
 
 pytestmark = pytest.mark.gpu
 
+N_BLOCKS = 64
+N_DW_ROWS = 256
 
-def _sample_blocks(batch, n, rng):
-    B = batch.T // batch.K
-    blocks = set(rng.choice(B, size=n, replace=False).tolist())
-    v = batch.valid.reshape(B, batch.K).bool()
-    partly = torch.nonzero((~v).any(1) & v.any(1)).squeeze(1)
-    if len(partly):
-        blocks.add(int(partly[0])); blocks.add(int(partly[-1]))        # masked blocks on purpose
+
+def oracle_forward_all_rows(cfg, batch):
+    """The oracle's forward state of every row: from the stored lse / label logits when they belong to
+    exactly these inputs, else computed now (minutes)."""
+    path = G.path_for(cfg)
+    if os.path.exists(path):
+        z = np.load(path)
+        dg = G.input_digests(batch)
+        if all(str(z["sha_" + k]) == dg[k] for k in ("H", "W", "labels", "valid")):
+            fwd = O.cat_forward_from_row_stats(z["lse"], z["z_label"], batch.labels, batch.valid, batch.K, batch.V)
+            assert fwd["n_valid"] == int(z["n_valid"]) and abs(fwd["loss"] - float(z["loss"])) <= 1e-12 * abs(float(z["loss"]))
+            return fwd
+        warnings.warn("config %d: the seeded inputs drawn here differ from the stored digests; running the oracle forward now" % cfg)
+    return O.cat_forward(batch.H, batch.W, batch.labels, batch.valid, batch.K, row_chunk=2048, check_rows_sum_to_one=False)
+
+
+def sample_blocks(batch, n, rng):
+    """>= n whole draft blocks: seeded random ones plus the kinds of block that must be covered."""
+    B, K = batch.T // batch.K, batch.K
+    blocks = set(rng.choice(B, size=n, replace=False).tolist()) | {0, B - 1}
+    v = batch.valid.reshape(B, K).bool().numpy()
+    tail = np.nonzero(~v[:, -1] & v[:, 0])[0]                           # block-end tail masked
+    hole = np.nonzero((~v[:, :-1] & v[:, 1:]).any(1))[0]                # masked row followed by a valid one
+    none = np.nonzero(~v.any(1))[0]                                     # fully masked
+    for kind in (tail, hole, none):
+        blocks.update(kind[:3].tolist()); blocks.update(kind[-1:].tolist())
     if batch.biased.any():
-        blocks.add(int(torch.nonzero(batch.biased)[0]) // batch.K)
-    blocks = sorted(blocks)
-    rows = np.concatenate([np.arange(b * batch.K, (b + 1) * batch.K) for b in blocks])
-    return rows
+        bb = np.unique(np.nonzero(batch.biased.numpy())[0] // K)
+        blocks.update(bb[:2].tolist()); blocks.update(bb[-1:].tolist())
+    blocks = np.array(sorted(blocks))
+    return (blocks[:, None] * K + np.arange(K)[None, :]).reshape(-1)
 
 
-def _check_any_size(batch, out, tol):
+def sample_vocab_rows(batch, n, rng):
+    """>= n token ids whose dW rows are compared."""
+    ok = O.effective_valid(batch.labels, batch.valid, batch.V)
+    counts = np.bincount(batch.labels.numpy()[ok], minlength=batch.V)
+    never = np.nonzero(counts == 0)[0]
+    last_tile = np.arange((batch.V - 1) // 256 * 256, batch.V)          # ragged last 256-column tile, if any
+    forced = np.concatenate([np.argsort(counts)[-28:], never[:24], never[-4:], [0, batch.V - 1],
+                             last_tile[:: max(1, len(last_tile) // 8)]])
+    return np.unique(np.concatenate([rng.choice(batch.V, n, replace=False), forced])), counts
+
+
+def check_any_size(batch, out):
     ok = O.effective_valid(batch.labels, batch.valid, batch.V)
     N = int(ok.sum())
     assert out["n_valid"] == N and out["status"] == 0
-    w32 = O.cat_weights_f32(out["conf"], ok, batch.K)
-    assert out["weight"].tobytes() == w32.tobytes()                      # bit-exact scan, all rows
-    ce = -np.log(out["conf"][ok].astype(np.float64))
-    loss64 = float((out["weight"][ok].astype(np.float64) * ce).sum() / N)
-    assert abs(out["loss"] - loss64) <= 1e-4 * abs(loss64)
-    col = np.abs(out["dW"].astype(np.float64).sum(axis=0)).max()
-    scale = np.abs(out["dW"].astype(np.float64)).sum(axis=0).max()
+    assert out["weight"].tobytes() == O.cat_weights_f32(out["conf"], ok, batch.K).tobytes()   # bit-exact scan, all rows
+    assert np.all(out["conf"][~ok] == 1.0) and np.all(out["weight"][~ok] == 0.0)
+    col = np.abs(out["dW"].sum(axis=0, dtype=np.float64)).max()
+    scale = np.abs(out["dW"]).sum(axis=0, dtype=np.float64).max()
     assert col <= 2e-3 * scale, (col, scale)                             # sum_v dz[r, v] = 0
     assert not out["dH"][~ok].any()
+    return N
 
 
-def _check_sampled(batch, out, rows, tol):
-    H_rows = batch.H[rows]
-    sub = synth.Batch(batch.spec, len(rows), batch.K, batch.d, batch.V, H_rows, batch.W, batch.labels[rows],
-                      batch.valid[rows], batch.biased[rows])
-    fwd = O.cat_forward(sub.H, sub.W, sub.labels, sub.valid, sub.K, row_chunk=256)
-    lse_err = np.max(np.abs(out["lse"][rows] - fwd["lse"]) / np.maximum(1.0, np.abs(fwd["lse"])))
-    assert lse_err <= tol["lse"], lse_err
-    cerr = np.max(np.abs(out["conf"][rows] - fwd["conf"]) / np.maximum(fwd["conf"], 1e-30))
-    assert cerr <= tol["conf"], cerr
-    werr = np.abs(out["weight"][rows].astype(np.float64) - fwd["weight"])
+def check_forward_all_rows(batch, out, fwd, tol):
+    assert abs(out["loss"] - fwd["loss"]) <= tol["loss"] * abs(fwd["loss"]), (out["loss"], fwd["loss"])
+    assert np.max(np.abs(out["lse"] - fwd["lse"]) / np.maximum(1.0, np.abs(fwd["lse"]))) <= tol["lse"]
+    cerr = np.abs(out["conf"] - fwd["conf"]) / np.maximum(fwd["conf"], 1e-30)
+    assert cerr.max() <= tol["conf"], (int(cerr.argmax()), cerr.max())
+    werr = np.abs(out["weight"].astype(np.float64) - fwd["weight"])
     assert np.all(werr <= batch.K * tol["conf"] * fwd["weight"] + 1e-37)
-    N = int(O.effective_valid(batch.labels, batch.valid, batch.V).sum())
-    dH = O.cat_dH_rows(sub.H, sub.W, sub.labels, fwd, np.arange(len(rows)), N)
-    assert rel_l2(out["dH"][rows], dH) <= tol["grad"], rel_l2(out["dH"][rows], dH)
-    first = np.arange(0, len(rows), batch.K)                              # position-0 rows carry most of the norm;
-    later = np.setdiff1d(np.arange(len(rows)), first)                     # check the other positions on their own
-    sure = np.exp(np.minimum(fwd["z_label"] - fwd["lse"], 0.0)) > 0.999
-    later = later[~sure[later]]
-    if np.linalg.norm(dH[later]) > 1e-30:
-        assert rel_l2(out["dH"][rows][later], dH[later]) <= 2 * tol["grad"]
 
 
-def _run(batch, fused):
+def run_path(batch, fused):
     dev = torch.device("cuda")
     H, W = batch.H.to(dev), batch.W.to(dev)
     y, valid = batch.labels.to(dev), batch.valid.to(dev)
@@ -92,43 +127,40 @@ def _run(batch, fused):
     return out
 
 
-@pytest.mark.parametrize("cfg,n_blocks", [(3, 6), (4, 12), (41, 12), (5, 4)])
-def test_full_size_sampled_blocks_and_invariants(cfg, n_blocks):
+@pytest.mark.parametrize("cfg", [2, 3, 4, 41, 5])
+def test_full_size_every_row_forward_sampled_dH_blocks_and_dW_rows(cfg):
     batch = synth.make_batch(cfg)
     tol = TOL[torch.bfloat16]
-    rows = _sample_blocks(batch, n_blocks, np.random.default_rng(cfg))
-    for fused in (True, False):
-        out = _run(batch, fused)
-        _check_any_size(batch, out, tol)
-        _check_sampled(batch, out, rows, tol)
-        del out
-
-
-def test_config2_full_size_whole_forward_and_sampled_dW_rows():
-    batch = synth.make_batch(2)
-    tol = TOL[torch.bfloat16]
-    fwd = O.cat_forward(batch.H, batch.W, batch.labels, batch.valid, batch.K, row_chunk=2048,
-                        check_rows_sum_to_one=False)
-    rng = np.random.default_rng(2)
-    counts = np.bincount(batch.labels.numpy(), minlength=batch.V)
-    vocab = np.unique(np.concatenate([rng.choice(batch.V, 200, replace=False), np.argsort(counts)[-28:],
-                                      np.nonzero(counts == 0)[0][:28], [0, batch.V - 1]]))
+    rng = np.random.default_rng(100 + cfg)
+    fwd = oracle_forward_all_rows(cfg, batch)
+    N = fwd["n_valid"]
+    rows = sample_blocks(batch, N_BLOCKS, rng)
+    assert len(rows) >= N_BLOCKS * batch.K
+    fwd_rows = {k: fwd[k][rows] for k in ("lse", "z_label", "weight", "eff_valid")}
+    dH_rows = O.cat_dH_rows(batch.H, batch.W, batch.labels, fwd_rows, rows, N)
+    vocab, counts = sample_vocab_rows(batch, N_DW_ROWS, rng)
+    assert len(vocab) >= N_DW_ROWS
     dW_rows = O.cat_dW_rows(batch.H, batch.W, batch.labels, fwd, vocab)
-    rows = _sample_blocks(batch, 8, rng)
+    w_norm_max = float(torch.linalg.vector_norm(batch.W.float(), dim=1).max())
+    row_norm = np.linalg.norm(dW_rows, axis=1)
     for fused in (True, False):
-        out = _run(batch, fused)
-        _check_any_size(batch, out, tol)
-        _check_sampled(batch, out, rows, tol)
-        assert abs(out["loss"] - fwd["loss"]) <= tol["loss"] * fwd["loss"]
-        assert np.max(np.abs(out["lse"] - fwd["lse"])) <= tol["lse"] * np.abs(fwd["lse"]).max()
-        assert rel_l2(out["dW"][vocab], dW_rows) <= tol["grad"], rel_l2(out["dW"][vocab], dW_rows)
+        out = run_path(batch, fused)
+        assert check_any_size(batch, out) == N
+        check_forward_all_rows(batch, out, fwd, tol)
+        g = out["dH"][rows]
+        assert rel_l2(g, dH_rows) <= tol["grad"], rel_l2(g, dH_rows)
+        check_dH_rows_by_position(g, dH_rows, fwd_rows, batch.K, w_norm_max, N, 1.0, tol["grad"])
+        got = out["dW"][vocab].astype(np.float64)
+        assert rel_l2(got, dW_rows) <= tol["grad"], rel_l2(got, dW_rows)
+        per_row = np.linalg.norm(got - dW_rows, axis=1) / np.maximum(row_norm, 1e-300)
+        live = row_norm > 1e-30
+        assert per_row[live].max() <= POSITION_FACTOR * tol["grad"], (fused, int(vocab[live][per_row[live].argmax()]), per_row[live].max())
         del out
 
 
 def test_config2_full_size_distillation_loss_sampled_blocks_and_invariants():
     """cat_kd_loss_fwd_bwd (Eq. 12) at the benchmark's size: a Llama-3.1-8B-shaped target head
     (d_t = 4096) over the T/K + K - 1 sequence positions the batch's blocks refer to."""
-    from paper_2605_08632_b200 import binding as B
     batch = synth.make_batch(2)
     ts = synth.make_target_side(batch, d_t=4096)
     tol = TOL[torch.bfloat16]
@@ -156,6 +188,6 @@ def test_config2_full_size_distillation_loss_sampled_blocks_and_invariants():
     g = cl.dH.float().cpu().numpy()[rows]
     assert rel_l2(g, dH_rows) <= tol["grad"], rel_l2(g, dH_rows)
     later = np.setdiff1d(np.arange(len(rows)), np.arange(0, len(rows), batch.K))
-    assert rel_l2(g[later], dH_rows[later]) <= 2 * tol["grad"]
+    assert rel_l2(g[later], dH_rows[later]) <= POSITION_FACTOR * tol["grad"]
     tot, ce, kd = cl.loss3.cpu().numpy()
     assert abs(tot - (beta * ce + kd)) <= 1e-6 * abs(tot) and kd > 0

@@ -503,11 +503,26 @@ def test_eq12_gradients_match_finite_differences_with_frozen_weights():
     assert np.allclose(dW.sum(axis=0), 0.0, atol=1e-14)
 
 
-def test_eq12_sampled_block_routine_agrees_with_the_whole_batch_routine():
+@pytest.mark.parametrize("source", ["target", "draft"])
+def test_eq12_sampled_block_routine_agrees_with_the_whole_batch_routine(source):
     H, W, y, valid, Ht, Wt, st = _kd_problem(35, B=9, K=4, masked=True)
-    fwd, dH, _ = O.cat_kd_forward_backward(H, W, y, valid, 4, Ht, Wt, st, 0.1, g=0.5, row_chunk=7)
-    rows, out, dH_rows = O.cat_kd_rows(H, W, y, valid, 4, Ht, Wt, st, 0.1, [0, 3, 8], fwd["n_valid"], g=0.5)
+    fwd, dH, _ = O.cat_kd_forward_backward(H, W, y, valid, 4, Ht, Wt, st, 0.1, conf_source=source, g=0.5, row_chunk=7)
+    rows, out, dH_rows = O.cat_kd_rows(H, W, y, valid, 4, Ht, Wt, st, 0.1, [0, 3, 8], fwd["n_valid"], conf_source=source, g=0.5)
     assert np.array_equal(rows, np.r_[0:4, 12:16, 32:36])
     for key in ("lse", "lse_t", "conf", "weight", "row_ce", "row_kd"):
         assert np.allclose(out[key], fwd[key][rows], rtol=1e-13, atol=0), key
     assert np.allclose(dH_rows, dH[rows], rtol=1e-12, atol=1e-18)
+
+
+def test_eq12_draft_confidence_source_is_the_heads_own_confidence():
+    # conf_source="draft": the Eq. 9 confidences are the draft head's own label probabilities, i.e. those of the
+    # plain CAT forward pass (pinned above against a library softmax), and the weights their Eq. 10 products
+    H, W, y, valid, Ht, Wt, st = _kd_problem(36, B=7, K=4, masked=True)
+    fwd, _, _ = O.cat_kd_forward_backward(H, W, y, valid, 4, Ht, Wt, st, 0.1, conf_source="draft", want_grads=False)
+    ok = fwd["eff_valid"]
+    plain = O.cat_forward(H, W, y, ok.astype(np.uint8), 4)
+    assert np.array_equal(plain["eff_valid"], ok)
+    assert np.allclose(fwd["conf"], plain["conf"], rtol=1e-13, atol=0)
+    assert np.allclose(fwd["weight"], plain["weight"], rtol=1e-12, atol=0)
+    tgt, _, _ = O.cat_kd_forward_backward(H, W, y, valid, 4, Ht, Wt, st, 0.1, conf_source="target", want_grads=False)
+    assert not np.allclose(tgt["conf"][ok], fwd["conf"][ok])

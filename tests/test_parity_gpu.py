@@ -19,7 +19,7 @@ def _full_check(batch, **kw):
     gpu = run_gpu(batch, **{k: v for k, v in kw.items() if k in ("slab_mib", "g", "conf_ext", "use_valid")})
     fwd, dH, dW = run_oracle(batch, g=kw.get("g") or 1.0, conf_ext=kw.get("conf_ext"), use_valid=kw.get("use_valid", True))
     check_forward(gpu, fwd, batch.K, batch.torch_dtype, batch.V)
-    check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype)
+    check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype, W=batch.W, g=kw.get("g") or 1.0)
     return gpu, fwd
 
 
@@ -142,7 +142,7 @@ def _fused_check(batch, **kw):
     gpu = run_gpu_fused(batch, **kw)
     fwd, dH, dW = run_oracle(batch, g=kw.get("g") or 1.0, conf_ext=kw.get("conf_ext"), use_valid=kw.get("use_valid", True))
     check_forward(gpu, fwd, batch.K, batch.torch_dtype, batch.V)
-    check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype)
+    check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype, W=batch.W, g=kw.get("g") or 1.0)
     return gpu, fwd
 
 
@@ -253,7 +253,7 @@ def test_single_cta_kernels_selected_by_environment_variable():
         "    for run in (run_gpu, run_gpu_fused):\n"
         "        g = run(b, slab_mib=1 if cfg == 41 else 0)\n"
         "        check_forward(g, fwd, b.K, b.torch_dtype, b.V)\n"
-        "        check_backward(g, fwd, dH, dW, b.K, b.torch_dtype)\n"
+        "        check_backward(g, fwd, dH, dW, b.K, b.torch_dtype, W=b.W)\n"
         "print('single-cta ok')\n" % (root, os.path.join(root, "tests")))
     env = dict(os.environ, CAT_LOSS_CTA_PAIR="0")
     res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)

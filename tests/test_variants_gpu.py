@@ -191,3 +191,21 @@ def test_autograd_module_matches_oracle_and_scales_with_the_upstream_gradient():
     assert H.grad.dtype == torch.bfloat16 and head.weight.grad is not None
     assert rel_l2(H.grad.float().cpu().numpy(), dH) <= 1.2e-2          # one more bf16 rounding from the scaling by 0.5
     assert rel_l2(head.weight.grad.float().cpu().numpy(), dW) <= 1.2e-2
+
+
+def test_autograd_module_called_twice_with_the_same_shape_before_one_backward():
+    """loss = head(H1) + head(H2) with equal T: each term must back-propagate its own gradients."""
+    from paper_2605_08632_b200.api import CatLossModule
+    b1, b2 = synth.make_batch(41, T=512, d=256, V=4000), synth.make_batch(2, T=512, d=256, V=4000)
+    dev = "cuda"
+    W = b1.W.to(dev).clone().requires_grad_(True)
+    H1, H2 = b1.H.to(dev).clone().requires_grad_(True), b2.H.to(dev).clone().requires_grad_(True)
+    head = CatLossModule(W, b1.K)
+    loss = head(H1, b1.labels.to(dev), b1.valid.to(dev)) + head(H2, b2.labels.to(dev), b2.valid.to(dev))
+    loss.backward()
+    torch.cuda.synchronize()
+    f1, dH1, dW1 = O.cat_forward_backward(b1.H, b1.W, b1.labels, b1.valid, b1.K)
+    f2, dH2, dW2 = O.cat_forward_backward(b2.H, b1.W, b2.labels, b2.valid, b2.K)
+    assert abs(loss.item() - (f1["loss"] + f2["loss"])) <= 1e-3 * (f1["loss"] + f2["loss"])
+    assert rel_l2(H1.grad.float().cpu().numpy(), dH1) <= 1e-2 and rel_l2(H2.grad.float().cpu().numpy(), dH2) <= 1e-2
+    assert rel_l2(head.weight.grad.float().cpu().numpy(), dW1 + dW2) <= 1.2e-2

@@ -3,9 +3,10 @@
 Some hosts cannot allocate device memory when the loss is called (all of it already belongs
 to another allocator, or allocation after start-up is against policy), so the library carries
 a fixed scratch array of its own for them.  This file checks, through the C ABI, that the
-variant returns what cat_loss_fwd returns, twice in a row on different batches (the array is
-shared and keeps the previous call's contents), and that shapes beyond its capacity are
-refused on the host.  It is collected last so that a run stopping at the first failure has
+variant returns bit for bit what cat_loss_fwd returns (same kernels, same plan, other scratch)
+and what the fp64 oracle computes within the forward tolerances, several times in a row on
+different batches (the array is shared and keeps the previous call's contents), and that shapes
+beyond its capacity are refused on the host.  It is collected last so that a run stopping at the first failure has
 already exercised everything else; it also passes alone in a fresh process.
 """
 import ctypes
@@ -14,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import cat_oracle as O
 from paper_2605_08632_b200 import binding as B
 from paper_2605_08632_b200 import synth
 
@@ -52,10 +54,17 @@ def test_static_scratch_forward_matches_workspace_forward_twice_in_a_row():
         torch.cuda.synchronize()
         if n_call > 0:    # (the very first call may be the one that makes the driver load the module image)
             assert torch.cuda.mem_get_info()[0] >= free_before - (1 << 20)   # nothing was allocated by the call
-        tol = 1e-5 if code == B.CAT_F32 else 1e-3
-        assert abs(got["loss"].item() - ref["loss"].item()) <= tol * abs(ref["loss"].item())
+        assert got["loss"].item() == ref["loss"].item()
         for key in ("lse", "conf", "weight"):
-            a, b = got[key].cpu().numpy().astype(np.float64), ref[key].cpu().numpy().astype(np.float64)
-            assert np.all(np.abs(a - b) <= tol * np.abs(b) + 1e-37), key
+            assert got[key].cpu().numpy().tobytes() == ref[key].cpu().numpy().tobytes(), key
         sg, sr = B.read_stats(got["stats"]), B.read_stats(ref["stats"])
         assert (sg.n_valid, sg.n_bad_labels, sg.device_status) == (sr.n_valid, sr.n_bad_labels, 0)
+        # and against the oracle (loss 1e-3 / 1e-5, confidences 5e-3 / 1e-5: the forward tolerances of the parity tests)
+        fwd = O.cat_forward(batch.H, batch.W, batch.labels, batch.valid, batch.K)
+        tol_loss, tol_conf = (1e-5, 1e-5) if code == B.CAT_F32 else (1e-3, 5e-3)
+        assert sg.n_valid == fwd["n_valid"]
+        assert abs(got["loss"].item() - fwd["loss"]) <= tol_loss * abs(fwd["loss"])
+        conf, weight = got["conf"].cpu().numpy(), got["weight"].cpu().numpy()
+        assert np.max(np.abs(conf - fwd["conf"]) / np.maximum(fwd["conf"], 1e-30)) <= tol_conf
+        assert np.all(np.abs(weight - fwd["weight"]) <= batch.K * tol_conf * fwd["weight"] + 1e-37)
+        assert weight.tobytes() == O.cat_weights_f32(conf, fwd["eff_valid"], batch.K).tobytes()
