@@ -12,7 +12,7 @@ Recording (the capture runs on a GPU machine, the CSV comes back, this runs on it un
     python bench.py --profile fused --config 2 --warmup 1 --steps 1          # plain run first, must exit 0
     ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --clock-control none \\
         -k regex:gemm_kernel --csv --log-file traffic_fused.csv python bench.py --profile fused --config 2 --warmup 1 --steps 1
-    python -m paper_2605_08632_b200.ncu_traffic record --workload config2 --rows 16384 --path fused traffic_fused.csv
+    python -m paper_2605_08632_b200.ncu_traffic record traffic_fused.csv --workload config2 --rows 16384 --path fused
 
 Launches are matched to stages by the kernel's template arguments (operand majors and epilogue)
 and taken from the LAST step in the capture, in launch order (row slab by row slab).
@@ -23,7 +23,6 @@ import csv
 import hashlib
 import json
 import os
-import sys
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 STORE = os.path.join(PKG_DIR, "ncu_traffic.json")
@@ -57,7 +56,8 @@ def parse(csv_path: str) -> list:
                 continue
             if hdr and len(r) == len(hdr):
                 d = dict(zip(hdr, r))
-                stage = next((s for frag, s in STAGE_OF.items() if frag in d["Kernel Name"]), None)
+                name = d["Kernel Name"].replace("cat::", "").replace("tc::", "")      # ncu may or may not print namespaces
+                stage = next((s for frag, s in STAGE_OF.items() if frag in name), None)
                 if stage is None:
                     continue
                 ent = launches.setdefault(int(d["ID"]), (stage, {}))
@@ -65,7 +65,7 @@ def parse(csv_path: str) -> list:
     return [launches[k] for k in sorted(launches)]
 
 
-def record(csv_path: str, workload: str, rows: int, path: str, launches_per_step: dict | None = None) -> dict:
+def record(csv_path: str, workload: str, rows: int, path: str) -> dict:
     per_stage = {}
     for stage, m in parse(csv_path):
         if "dram__bytes_read.sum" in m and "dram__bytes_write.sum" in m:
