@@ -191,14 +191,17 @@ def time_config(cfg_id, dev, local_rank, warmup=3, steps=5):
 
 def nccl_summary(log_dir):
     """What NCCL's own log says about the transport (NVLS, rings/trees), from the per-rank debug files."""
-    out = {"nvls": False, "lines": []}
+    out = {"nvls": False, "files": 0, "log_lines": 0, "lines": []}
+    keys = ("NCCL version", "NVLS", "Connected all", "Channel 00", "via P2P", "via SHM", "Using network", "comm 0x")
     try:
         for fn in sorted(os.listdir(log_dir)):
+            out["files"] += 1
             with open(os.path.join(log_dir, fn), errors="replace") as f:
                 for line in f:
-                    if "NVLS" in line:
+                    out["log_lines"] += 1
+                    if "NVLS" in line and "disabled" not in line.lower():
                         out["nvls"] = True
-                    if any(k in line for k in ("NCCL version", "NVLS multicast support", "Connected all", "comm 0x")) and len(out["lines"]) < 8:
+                    if any(k in line for k in keys) and len(out["lines"]) < 10:
                         out["lines"].append(line.strip()[-160:])
     except Exception as e:      # the summary is an extra: never fail the run for it
         out["error"] = repr(e)
