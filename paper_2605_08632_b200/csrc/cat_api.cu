@@ -129,6 +129,30 @@ BwdPlan plan_bwd(const cat_shape* s) {
     if (Vs > v_pad) Vs = v_pad;
     p.n_slabs = static_cast<int>(cdiv(s->V, Vs));
     p.Vs = cdiv(cdiv(s->V, p.n_slabs), 256) * 256;      // rebalance the slabs
+    if (s->in_dtype == CAT_BF16) {
+        // Among slab widths within the budget take the one whose dW GEMMs (tiles of a slab = vocabulary tiles x
+        // d/256, one per worker at a time) need the fewest waves in total, charging one wave per slab for its
+        // fixed costs (launches, one more pass over the fp32 dH accumulator).  A slab of 32 vocabulary tiles at
+        // d = 3072 is 384 tiles = 5.2 waves of 74 and pays for 6; 30 tiles is 4.9 and pays for 5.
+        const long long n_tiles_n = cdiv(s->d, tc::BN);
+        long long best_vs = p.Vs, best_cost = -1;
+        for (long long vs = Vs, tries = 0; vs >= 256 && tries < 128; vs -= 256, ++tries) {
+            long long cost = 0;
+            for (long long v0 = 0; v0 < s->V; v0 += vs) {
+                const long long w = (s->V - v0) < vs ? (s->V - v0) : vs;
+                cost += cdiv(cdiv(w, tile_m()) * n_tiles_n, plan_workers()) + 1;
+            }
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_vs = vs; }
+        }
+        {   // the even split above, if it is at least as good
+            long long cost = 0;
+            for (long long v0 = 0; v0 < s->V; v0 += p.Vs) {
+                const long long w = (s->V - v0) < p.Vs ? (s->V - v0) : p.Vs;
+                cost += cdiv(cdiv(w, tile_m()) * n_tiles_n, plan_workers()) + 1;
+            }
+            if (cost > best_cost) p.Vs = best_vs;
+        }
+    }
     p.n_slabs = static_cast<int>(cdiv(s->V, p.Vs));
     size_t off = kHeaderBytes;
     p.off_dz = off; off = align256(off + elt * static_cast<size_t>(s->T) * p.Vs);
