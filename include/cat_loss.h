@@ -81,7 +81,7 @@ typedef struct {
                           fp32 accumulation.  CAT_F32: fp32 FFMA path, fp32 throughout */
     int32_t dW_dtype;  /* cat_dtype of dW: CAT_F32 (default) or CAT_BF16 (bf16 inputs only) */
     int32_t slab_mib;  /* cap, in MiB, on the large scratch slab (dz slab of cat_loss_bwd,
-                          logits slab of cat_loss_fwd_bwd); 0 = default (2048 / 2560).
+                          logits slab of cat_loss_fwd_bwd); 0 = default (2048 / 3072).
                           Smaller caps mean more, smaller slabs.                          */
     int64_t ldH;       /* row pitch of H and dH in elements, >= d                     */
     int64_t ldW;       /* row pitch of W and dW in elements, >= d                     */
@@ -199,7 +199,7 @@ int cat_count_valid(const cat_shape* shape, const int64_t* labels, const uint8_t
  * epilogue, the dW GEMM takes a[r] * H[r, :] as its second operand, and no second pass over the slab
  * is needed.  dH is written once per slab, dW accumulated over slabs in fp32.  Executed work is the
  * 6*T*d*V flops of the three contractions instead of 8*T*d*V; the price is one slab of 16-bit values
- * in the workspace (at most about slab_mib MiB, default 2560, and always at least two slabs once T
+ * in the workspace (at most about slab_mib MiB, default 3072, and always at least two slabs once T
  * exceeds one slab unit, so a T x V matrix never exists at once) and bf16 rounding of the stored
  * numerators (relative 2^-9, the same as rounding dz to bf16).  e is formed as exp(z - m) * exp(m - ref),
  * m the running row maximum, with m - ref capped at 79.7 so that e stays finite for any input: only a

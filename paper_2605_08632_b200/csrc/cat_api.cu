@@ -28,7 +28,7 @@ constexpr size_t kHeaderBytes = 256;     // workspace header: int32 status at by
 constexpr size_t kScaleOffset = 64;
 constexpr int kMaxSplits = 128;
 constexpr long long kDefaultSlabMiB = 2048;
-constexpr long long kDefaultFusedSlabMiB = 2560;
+constexpr long long kDefaultFusedSlabMiB = 3072;
 
 inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 inline long long cdiv(long long a, long long b) { return (a + b - 1) / b; }
@@ -186,20 +186,24 @@ FusedPlan plan_fused(const cat_shape* s) {
     const long long most = ((s->T - 1) / L) * L;                // at least two slabs: the T x V logits never coexist
     if (most >= L && cap > most) cap = most;
     if (cap < L) cap = L;
-    // among slab heights within the budget, take the one with the fewest waves of dH tiles
-    // (tiles per slab = m-tiles * d/256, one per worker at a time), then the fewest slabs
-    const long long n_tiles_n = cdiv(s->d, tc::BN);
+    // Among slab heights within the budget take the one that costs the three GEMMs the fewest tile-steps
+    // (waves of the 74 tile-workers x k-slices per tile, summed over the slabs): the logits GEMM (items are
+    // runs of vocabulary tiles, see fwd_splits), dH (row tiles x d/256 tiles, the whole vocabulary contracted)
+    // and dW (vocabulary tiles x d/256 tiles, the slab's rows contracted).  Ties go to the taller slab.
+    const long long n_tiles_n = cdiv(s->d, tc::BN), n_tiles_v = cdiv(s->V, tc::BN);
     long long best_ts = cap;
-    long long best_waves = -1, best_slabs = 0;
+    double best_cost = -1.0;
     for (long long ts = cap, tries = 0; ts >= L && tries < 96; ts -= L, ++tries) {
-        long long waves = 0, slabs = 0;
-        for (long long r0 = 0; r0 < s->T; r0 += ts, ++slabs) {
+        double cost = 0.0;
+        for (long long r0 = 0; r0 < s->T; r0 += ts) {
             const long long rws = (s->T - r0) < ts ? (s->T - r0) : ts;
-            waves += cdiv(cdiv(rws, tile_m()) * n_tiles_n, plan_workers());
+            const long long num_m = cdiv(rws, tile_m());
+            const long long S = fwd_splits(rws, s->V);
+            cost += static_cast<double>(cdiv(num_m * S, plan_workers()) * cdiv(n_tiles_v, S)) * static_cast<double>(s->d);   // logits
+            cost += static_cast<double>(cdiv(num_m * n_tiles_n, plan_workers())) * static_cast<double>(s->V);               // dH
+            cost += static_cast<double>(cdiv(n_tiles_v * n_tiles_n, plan_workers())) * static_cast<double>(rws);             // dW
         }
-        if (best_waves < 0 || waves < best_waves || (waves == best_waves && slabs < best_slabs)) {
-            best_waves = waves; best_slabs = slabs; best_ts = ts;
-        }
+        if (best_cost < 0.0 || cost < best_cost * (1.0 - 1e-9)) { best_cost = cost; best_ts = ts; }
     }
     p.Ts = best_ts;
     p.n_slabs = static_cast<int>(cdiv(s->T, p.Ts));
