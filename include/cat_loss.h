@@ -24,9 +24,10 @@
  * General conventions
  *   - Every data pointer is a DEVICE pointer owned by the caller, valid on the current
  *     device, unless a parameter says "host".  cat_shape is read on the host.
- *   - Nothing is allocated or freed here and no state is kept between calls.  The one exception is
- *     cat_loss_fwd_static, which owns a fixed device array inside the library image and remembers,
- *     per device, that array's address (see there).
+ *   - Nothing is allocated or freed here and no state is kept between calls, with two exceptions:
+ *     cat_loss_fwd_static owns a fixed device array inside the library image and remembers, per
+ *     device, that array's address (see there); and the first tensor-core GEMM on a device measures
+ *     which SMs share an L2 partition and keeps the result in the library image (see cat_die_map).
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *     stream) and the call returns without synchronising.
  *   - Argument errors that the host can see return a negative cat_status before anything is
@@ -390,6 +391,24 @@ int cat_kd_loss_fwd_bwd(const cat_shape* shape, const cat_kd_desc* desc, const v
  * pass.  Host-only; returns 0 for an invalid shape.
  */
 int cat_loss_launch_count(const cat_shape* shape, int pass);
+
+/*
+ * What the library has measured about the current device's two L2 partitions (no counterpart in the
+ * paper: it concerns how this library's GEMM kernels are placed on a B200).  The first tensor-core GEMM
+ * launched on a device is preceded, on the same stream, by two small kernels (about 0.2 ms, once per device
+ * and process, skipped while the stream is being captured) that time atomics from every SM and sort the SMs
+ * into the two dies; the persistent GEMM kernels then number their CTA pairs die by die, because
+ * neighbouring pairs share operand tiles and a tile shared across the dies is fetched into both L2
+ * partitions.  Results do not depend on it (every pair claims its index with an atomic and falls back to
+ * the next free one); DRAM traffic and time do.  This call runs the measurement if it has not run yet,
+ * WAITS for `cuda_stream`, and reports the table:
+ *   worker_of_tpc  HOST array of `capacity` int32, or NULL: entry t is the worker index suggested to the CTA
+ *                  pair running on SMs 2t and 2t+1                                             (host, out)
+ *   n_first_die    HOST int32, or NULL: number of TPCs on the die of SM 0                       (host, out)
+ * Returns the number of TPCs the table covers (74 on a full B200), 0 if the measurement was not clean
+ * enough to be used (the kernels then number their pairs by blockIdx), or a negative cat_status.
+ */
+int cat_die_map(int32_t* worker_of_tpc, int capacity, int32_t* n_first_die, void* cuda_stream);
 
 /*
  * Self-test of the error path that cat_stats.device_status / the workspace status word report (no

@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.cat_kd_workspace_bytes.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc), vp]
         L.cat_kd_loss_fwd_bwd.restype = ctypes.c_int
         L.cat_kd_loss_fwd_bwd.argtypes = [ctypes.POINTER(cat_shape), ctypes.POINTER(cat_kd_desc)] + [vp] * 16 + [ctypes.c_int, vp, sz, vp]
+        L.cat_die_map.restype = ctypes.c_int
+        L.cat_die_map.argtypes = [vp, ctypes.c_int, vp, vp]
         L.cat_selftest_wait_timeout.restype = ctypes.c_int
         L.cat_selftest_wait_timeout.argtypes = [ctypes.c_int, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp]
         _lib = L
@@ -265,6 +267,17 @@ def cat_kd_loss_fwd_bwd(shape, desc, H, W, labels, valid, Ht, Wt, block_start_ho
                                    workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream())
     if rc != CAT_OK:
         raise CatError(rc, "cat_kd_loss_fwd_bwd")
+
+
+def cat_die_map():
+    """(worker_of_tpc list, TPCs on the die of SM 0) as measured on the current device, or ([], 0) when the
+    measurement could not be used.  Waits for the current stream."""
+    arr = (ctypes.c_int32 * 128)()
+    n0 = ctypes.c_int32(0)
+    n = lib().cat_die_map(arr, 128, ctypes.byref(n0), _stream())
+    if n < 0:
+        raise CatError(n, "cat_die_map")
+    return list(arr[:n]), int(n0.value)
 
 
 def cat_selftest_wait_timeout(role: int, short_ns: int, long_ns: int, status, elapsed_ns) -> None:

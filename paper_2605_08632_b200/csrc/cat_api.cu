@@ -12,6 +12,7 @@
 
 #include <math.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "kd.cuh"
@@ -19,12 +20,22 @@
 #include "simt.cuh"
 #include "tc_gemm.cuh"
 
+// ------------------------------------------------------------------------------------------
+// Forward pass with built-in scratch, for callers that may not allocate device memory.
+// The array below is part of the module image: each GPU that loads the library carries it
+// until the process ends.  Host code must not use the symbol's name as a pointer (on the host
+// it is only a stand-in); the device address is fetched once per device with
+// cudaGetSymbolAddress and that address is what the kernels receive.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[CAT_STATIC_SCRATCH_BYTES];
+
 namespace {
 
 using namespace cat;
 
 constexpr int kPlanSMs = 148;            // B200: the static schedules are planned for 148 SMs
-constexpr size_t kHeaderBytes = 256;     // workspace header: int32 status at byte 0, fp32 g/N at byte 64
+constexpr size_t kHeaderBytes = 1024;    // workspace header: int32 status at byte 0, fp32 g/N at byte 64, worker claims from byte 256
+constexpr size_t kClaimsOffset = 256;    // up to 192 ints: one per CTA pair of a GEMM launch
 constexpr size_t kScaleOffset = 64;
 constexpr int kMaxSplits = 128;
 constexpr long long kDefaultSlabMiB = 2048;
@@ -383,9 +394,72 @@ int band_tiles(long long d) {
     return static_cast<int>(b < 1 ? 1 : b);
 }
 
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// Set-up, once per device, with that device current: resolve the array's device address.
+int static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_ARCH; }
+    if (dev < 0 || dev >= kMaxDevices) return CAT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return CAT_ERR_CUDA; }
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return CAT_OK;
+}
+void* static_scratch_base() {
+    void* p = nullptr;
+    return static_scratch_address(&p) == CAT_OK ? p : nullptr;
+}
+
+// The device's die map (diemap.cuh) is measured by the first GEMM launch on each device, on that launch's
+// stream, ahead of the GEMM: two small kernels, about 0.2 ms, nothing allocated (the lines they time lie in
+// the library's built-in scratch array, whose contents they leave as they are), no synchronisation.  Kernels
+// that run before the table is final number their workers by blockIdx.  Skipped while the stream is being
+// captured (it would be replayed with every graph launch) and tried again on the next call.
+std::mutex g_die_mu;
+bool g_die_launched[64] = {};
+
+void ensure_die_map(int sm_count, cudaStream_t st) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return; }
+    std::lock_guard<std::mutex> lock(g_die_mu);
+    if (g_die_launched[dev]) return;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) { cudaGetLastError(); return; }
+    static const bool off = [] { const char* e = getenv("CAT_LOSS_DIE_MAP"); return e && e[0] == '0'; }();     // CAT_LOSS_DIE_MAP=0: number the pairs by blockIdx
+    void* base = off ? nullptr : static_scratch_base();
+    if (!base || sm_count > die::MAX_SM) { g_die_launched[dev] = true; return; }      // no table: blockIdx order stays
+    // N_LINES lines about 1 MiB apart (a whole number of 128-byte lines), all inside the array
+    const size_t stride_words = static_cast<size_t>(CAT_STATIC_SCRATCH_BYTES) / 4 / die::N_LINES - 64;
+    die::probe_kernel<<<sm_count * 8, 32, 0, st>>>(static_cast<unsigned*>(base), stride_words, sm_count);
+    die::classify_kernel<<<1, 32, 0, st>>>(sm_count);
+    cudaGetLastError();
+    g_die_launched[dev] = true;
+}
+
+unsigned next_launch_serial() {
+    static std::atomic<unsigned> n{0};
+    unsigned v = ++n;
+    v &= 0x7fffffffu;
+    return v == 0 ? ++n & 0x7fffffffu : v;
+}
+
 template <int A_MN, int B_MN, class Epi, int CG>
-int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const tc::Sched& sched,
+int launch_tc_cg(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const tc::Sched& sched_in,
                  const typename Epi::Params& ep, int* status, int sm_count, cudaStream_t st) {
+    tc::Sched sched = sched_in;
+    if (CG == 2) {
+        ensure_die_map(sm_count, st);
+        sched.claims = status + kClaimsOffset / sizeof(int);        // `status` is the first word of a workspace header
+        sched.serial = static_cast<int>(next_launch_serial());
+    }
     auto kern = tc::gemm_kernel<A_MN, B_MN, Epi, CG>;
     constexpr int smem = tc::Geo<CG>::SMEM_BYTES;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -448,6 +522,8 @@ tc::Sched make_sched(long long M, long long N, long long Kd, int n_groups, int b
     s.n_fastest = n_fastest;
     s.n_items = s.num_m_tiles * s.n_groups;
     s.wait_ns = tc::WAIT_LIMIT_NS;
+    s.claims = nullptr;
+    s.serial = 0;
     return s;
 }
 
@@ -1090,36 +1166,6 @@ int cat_conf_window(const float* conf_seq, int64_t L, const int64_t* block_start
     return cudaGetLastError() == cudaSuccess ? CAT_OK : CAT_ERR_CUDA;
 }
 
-// ------------------------------------------------------------------------------------------
-// Forward pass with built-in scratch, for callers that may not allocate device memory.
-// The array below is part of the module image: each GPU that loads the library carries it
-// until the process ends.  Host code must not use the symbol's name as a pointer (on the host
-// it is only a stand-in); the device address is fetched once per device with
-// cudaGetSymbolAddress and that address is what the kernels receive.
-// ------------------------------------------------------------------------------------------
-static __device__ __align__(256) unsigned char g_static_scratch[CAT_STATIC_SCRATCH_BYTES];
-
-namespace {
-constexpr int kMaxDevices = 64;
-std::mutex g_static_mu;
-void* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
-
-// Set-up, once per device, with that device current: resolve the array's device address.
-int static_scratch_address(void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_ARCH; }
-    if (dev < 0 || dev >= kMaxDevices) return CAT_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(g_static_mu);
-    if (!g_static_ptr[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return CAT_ERR_CUDA; }
-        g_static_ptr[dev] = p;
-    }
-    *out = g_static_ptr[dev];
-    return CAT_OK;
-}
-}  // namespace
-
 int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W, const int64_t* labels, const uint8_t* valid,
                         const float* conf_ext, float* loss, float* lse, float* conf, float* weight, cat_stats* stats,
                         void* cuda_stream) {
@@ -1139,6 +1185,21 @@ int cat_loss_fwd_static(const cat_shape* shape, const void* H, const void* W, co
     // in the scratch is fully rewritten before it is read
     return cat_loss_fwd(shape, H, W, labels, valid, conf_ext, loss, lse, conf, weight, stats, scratch,
                         static_cast<size_t>(CAT_STATIC_SCRATCH_BYTES), cuda_stream);
+}
+
+int cat_die_map(int32_t* worker_of_tpc, int capacity, int32_t* n_first_die, void* cuda_stream) {
+    int sms = 0;
+    const int dc = check_device(&sms);
+    if (dc != CAT_OK) return dc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ensure_die_map(sms, st);
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    die::Map m;
+    if (cudaMemcpyFromSymbol(&m, die::g_map, sizeof(m)) != cudaSuccess) { cudaGetLastError(); return CAT_ERR_CUDA; }
+    if (m.valid != 1 || m.n_tpc <= 0 || m.n_tpc > die::MAX_SM / 2) return 0;
+    for (int t = 0; worker_of_tpc && t < m.n_tpc && t < capacity; ++t) worker_of_tpc[t] = m.worker_of_tpc[t];
+    if (n_first_die) *n_first_die = m.n_die0;
+    return m.n_tpc;
 }
 
 }  // extern "C"

@@ -17,6 +17,7 @@
 // CAT_ERR_TIMEOUT in the status word, drains what it issued, frees its TMEM and returns.
 #pragma once
 #include "ptx.cuh"
+#include "diemap.cuh"
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -46,6 +47,8 @@ struct Sched {
     int n_fastest;     // 1: items ordered group-fastest within an m-tile; 0: m-fastest within (band, group)
     int n_items;       // num_m_tiles * n_groups
     unsigned long long wait_ns;   // limit of every mbarrier wait in the kernel
+    int* claims;       // CTA pairs: worker indices taken in this launch (>= gridDim.x / 2 ints), or nullptr = blockIdx order
+    int serial;        // this launch's mark in `claims`, unique per launch and not 0
 };
 
 __device__ __forceinline__ void decode_item(const Sched& s, int item, int& m_tile, int& group, int& n_begin, int& n_end) {
@@ -71,6 +74,7 @@ struct Ctl {
     unsigned long long tempty[2];
     unsigned long long drain;
     uint32_t tmem_base;
+    uint32_t worker;
     volatile int abort;
 };
 
@@ -555,15 +559,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int lane = threadIdx.x & 31;
     const uint32_t rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
     const bool leader = rank == 0;
-    const int worker = blockIdx.x / CG;          // a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
-    const int n_workers = gridDim.x / CG;
+    const int n_workers = gridDim.x / CG;        // a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
+    int worker = blockIdx.x / CG;
+    const bool claimed = CG == 2 && sched.claims != nullptr;
 
     if (threadIdx.x == 0) {
         ptx::prefetch_tmap(&tmA);
         ptx::prefetch_tmap(&tmB);
         ptx::prefetch_tmap(&tmOut);
+        // pairs are numbered die by die where the device's map is known (neighbouring workers share operand tiles)
+        if (claimed && leader) ctl.worker = static_cast<uint32_t>(die::claim_worker(sched.claims, sched.serial, worker, n_workers));
     }
     cta_begin<CG>(ctl, G::STAGES, warp);
+    if (claimed) worker = static_cast<int>(leader ? ctl.worker : ptx::ld_shared_cluster_u32(ptx::mapa_shared(ptx::smem_u32(&ctl.worker), 0)));
     const uint32_t tmem = ctl.tmem_base;
     volatile int* abort = &ctl.abort;
     const unsigned long long wait_ns = sched.wait_ns;

@@ -1,0 +1,35 @@
+"""The measured SM-to-die table that the GEMM kernels number their CTA pairs by: on a B200 it must be a
+permutation of the pair indices with both dies populated; and whatever it says, results are those of the
+oracle (the kernels claim worker indices with atomics, so the table is advice only)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_08632_b200 import binding as B
+from paper_2605_08632_b200 import synth
+
+from parity_util import check_backward, check_forward, run_gpu, run_gpu_fused, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def test_die_map_is_a_permutation_with_two_populated_dies():
+    table, n0 = B.cat_die_map()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert len(table) == sms // 2, "the measurement was not usable on this device"
+    assert sorted(table) == list(range(len(table)))
+    assert len(table) // 4 <= n0 <= 3 * len(table) // 4
+    # the first n0 worker indices belong to the die of SM 0, and TPC 0 is on it
+    assert table[0] < n0
+    again, n0b = B.cat_die_map()
+    assert again == table and n0b == n0                       # measured once per device and process
+
+
+def test_full_grid_gemms_match_the_oracle_with_the_table_in_use():
+    # enough rows and columns that every GEMM launches all 74 CTA pairs, several items each
+    batch = synth.make_batch(41, T=20480, d=512, V=20480)
+    fwd, dH, dW = run_oracle(batch)
+    for run in (run_gpu, run_gpu_fused):
+        gpu = run(batch)
+        check_forward(gpu, fwd, batch.K, batch.torch_dtype, batch.V)
+        check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype, W=batch.W)
