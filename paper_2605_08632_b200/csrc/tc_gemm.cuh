@@ -581,13 +581,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, issued = 0;
             bool ok = true;
+            // Consecutive tiles walk the contraction in opposite directions: an operand that every tile re-reads
+            // from start to end (the scaled H rows in dW, 39 MB at config 2, next to the streaming slab) is then
+            // met again most-recent-lines first, which an LRU cache can serve, instead of oldest first, which it
+            // cannot once the footprint exceeds it.  dW read 4.6 GB per launch one way only, 3.7 GB this way.
+            // (The sum over k is taken in another order in every other tile: still fixed, run to run.)
+            uint32_t rev = 0;
             for (int item = worker; item < sched.n_items && ok; item += n_workers) {
                 int m_tile, group, n_begin, n_end;
                 decode_item(sched, item, m_tile, group, n_begin, n_end);
                 const int m0 = (m_tile * CG + static_cast<int>(rank)) * BM;
-                for (int n = n_begin; n < n_end && ok; ++n) {
+                for (int n = n_begin; n < n_end && ok; ++n, rev ^= 1u) {
                     const int n0 = n * BN + static_cast<int>(rank) * G::BN_CTA;
-                    for (int kb = 0; kb < sched.num_kb; ++kb) {
+                    for (int kbi = 0; kbi < sched.num_kb; ++kbi) {
+                        const int kb = rev ? sched.num_kb - 1 - kbi : kbi;
                         if (!wait_bounded(ptx::smem_u32(&ctl.empty[stage]), phase ^ 1u, abort, status, wait_ns)) { ok = false; break; }
                         const uint32_t full_local = ptx::smem_u32(&ctl.full[stage]);
                         if (leader) ptx::mbar_arrive_expect_tx(full_local, G::STAGE_BYTES * CG);
