@@ -33,3 +33,38 @@ def test_full_grid_gemms_match_the_oracle_with_the_table_in_use():
         gpu = run(batch)
         check_forward(gpu, fwd, batch.K, batch.torch_dtype, batch.V)
         check_backward(gpu, fwd, dH, dW, batch.K, batch.torch_dtype, W=batch.W)
+
+
+def _digest_code(root):
+    return (
+        "import sys, hashlib; sys.path.insert(0, %r)\n"
+        "import torch\n"
+        "from paper_2605_08632_b200 import synth, binding as B\n"
+        "from paper_2605_08632_b200.api import CatLoss\n"
+        "b = synth.make_batch(41, T=20480, d=512, V=20480)\n"
+        "dev = 'cuda'\n"
+        "cl = CatLoss(b.T, b.d, b.V, b.K)\n"
+        "args = (b.H.to(dev), b.W.to(dev), b.labels.to(dev), b.valid.to(dev))\n"
+        "h = hashlib.sha256()\n"
+        "cl.forward_backward(*args); torch.cuda.synchronize()\n"
+        "for t in (cl.lse, cl.weight, cl.dH.view(torch.int16), cl.dW): h.update(t.cpu().numpy().tobytes())\n"
+        "cl.forward(*args); cl.backward(*args); torch.cuda.synchronize()\n"
+        "for t in (cl.lse, cl.weight, cl.dH.view(torch.int16), cl.dW): h.update(t.cpu().numpy().tobytes())\n"
+        "print('DIGEST', h.hexdigest(), len(B.cat_die_map()[0]))\n" % root)
+
+
+def test_results_are_bitwise_the_same_with_and_without_the_table():
+    """CAT_LOSS_DIE_MAP=0 (read once per process, hence the children) leaves the CTA pairs numbered by blockIdx."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = {}
+    for flag in ("1", "0"):
+        env = dict(os.environ, CAT_LOSS_DIE_MAP=flag)
+        res = subprocess.run([sys.executable, "-c", _digest_code(root)], env=env, capture_output=True, text=True, timeout=900)
+        assert res.returncode == 0 and "DIGEST" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
+        _, digest, n = res.stdout.strip().splitlines()[-1].split()
+        out[flag] = (digest, int(n))
+    assert out["0"][1] == 0 and out["1"][1] > 0          # the switch really turned the table off / it was measured
+    assert out["0"][0] == out["1"][0]
