@@ -573,6 +573,9 @@ def main():
     per_step = B.cat_loss_launch_count(cl.shape, 2)
     out["gpu_launches"] = per_step * args.steps * world
     out["launches_per_step"] = per_step
+    table, n_first = B.cat_die_map()
+    out["die_map"] = {"tpcs": len(table), "tpcs_on_first_die": n_first,
+                      "what": "SM-to-die table measured by the library on this device; the GEMM kernels number their CTA pairs by it (0 tpcs: not usable, blockIdx order)"}
     if dist is not None:
         out["nccl"] = nccl_summary(nccl_dir)
 
