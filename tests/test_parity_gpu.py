@@ -276,3 +276,28 @@ def test_seeded_random_shapes_both_paths():
             gpu = run(batch, slab_mib=slab)
             check_forward(gpu, fwd, K, batch.torch_dtype, V)
             check_backward(gpu, fwd, dH, dW, K, batch.torch_dtype, per_position=False)
+
+
+def test_non_finite_inputs_propagate_without_a_trap():
+    """A NaN or an infinity in H is not treated specially: the row's statistics, the rows after it in its draft
+    block (their weights contain its confidence), the loss and dW come out non-finite; rows of other blocks are
+    what they would have been; the kernels finish, report no device error, and the context stays usable."""
+    batch = synth.make_batch(2, T=256, d=128, V=1000)
+    clean = {False: run_gpu(batch), True: run_gpu_fused(batch)}
+    batch.H[17, 5] = float("nan")
+    batch.H[40, 3] = float("inf")
+    others = np.setdiff1d(np.arange(batch.T), np.r_[16:24, 40:48])
+    for fused, run in ((False, run_gpu), (True, run_gpu_fused)):
+        gpu = run(batch)
+        assert gpu["stats"].device_status == 0 and gpu["bwd_status"] == 0
+        assert not np.isfinite(gpu["lse"][17]) and not np.isfinite(gpu["lse"][40])
+        assert not np.isfinite(gpu["loss"])
+        assert not np.isfinite(gpu["dH"][17]).all() and not np.isfinite(gpu["dH"][40]).all()
+        assert not np.isfinite(gpu["weight"][18:24]).any() and not np.isfinite(gpu["weight"][41:48]).any()
+        assert not np.isfinite(gpu["dW"]).all()
+        for key in ("lse", "conf", "weight"):
+            assert gpu[key][others].tobytes() == clean[fused][key][others].tobytes(), key
+        assert np.isfinite(gpu["dH"][others]).all()
+        assert rel_l2(gpu["dH"][others], clean[fused]["dH"][others]) <= 1e-6
+    again = run_gpu(synth.make_batch(2, T=256, d=128, V=1000))
+    assert again["lse"].tobytes() == clean[False]["lse"].tobytes() and np.isfinite(again["dW"]).all()
