@@ -141,7 +141,7 @@ BwdPlan plan_bwd(const cat_shape* s) {
     p.n_slabs = static_cast<int>(cdiv(s->V, Vs));
     p.Vs = cdiv(cdiv(s->V, p.n_slabs), 256) * 256;      // rebalance the slabs
     if (s->in_dtype == CAT_BF16) {
-        // Among slab widths within the budget take the one whose dW GEMMs (tiles of a slab = vocabulary tiles x
+        // Among slab widths within the cap take the one whose dW GEMMs (tiles of a slab = vocabulary tiles x
         // d/256, one per worker at a time) need the fewest waves in total, charging one wave per slab for its
         // fixed costs (launches, one more pass over the fp32 dH accumulator).  A slab of 32 vocabulary tiles at
         // d = 3072 is 384 tiles = 5.2 waves of 74 and pays for 6; 30 tiles is 4.9 and pays for 5.
@@ -193,11 +193,11 @@ FusedPlan plan_fused(const cat_shape* s) {
     p.ldz = cdiv(s->V, 256) * 256;
     const long long L = (static_cast<long long>(s->K) * tile_m()) / gcd_ll(s->K, tile_m());   // lcm(K, rows per m-tile)
     const long long mib = s->slab_mib > 0 ? s->slab_mib : kDefaultFusedSlabMiB;
-    long long cap = ((mib << 20) / (p.ldz * 2) / L) * L;       // rows that fit the slab budget
+    long long cap = ((mib << 20) / (p.ldz * 2) / L) * L;       // rows that fit the slab cap
     const long long most = ((s->T - 1) / L) * L;                // at least two slabs: the T x V logits never coexist
     if (most >= L && cap > most) cap = most;
     if (cap < L) cap = L;
-    // Among slab heights within the budget take the one that costs the three GEMMs the fewest tile-steps
+    // Among slab heights within the cap take the one that costs the three GEMMs the fewest tile-steps
     // (waves of the 74 tile-workers x k-slices per tile, summed over the slabs): the logits GEMM (items are
     // runs of vocabulary tiles, see fwd_splits), dH (row tiles x d/256 tiles, the whole vocabulary contracted)
     // and dW (vocabulary tiles x d/256 tiles, the slab's rows contracted).  Ties go to the taller slab.

@@ -7,7 +7,7 @@ file together with a digest of the kernel sources they were taken from.  `load()
 numbers out only while the sources still have that digest: once a kernel changes, the traffic
 figure is gone (None) until a new capture is recorded.
 
-Recording (the capture runs on a GPU machine, the CSV comes back, this runs on it unchanged sources):
+Recording (run the capture on a machine with a B200, then this tool on its CSV, with the sources unchanged in between):
 
     python bench.py --profile fused --config 2 --warmup 1 --steps 1          # plain run first, must exit 0
     ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --clock-control none \\
